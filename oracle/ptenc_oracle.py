@@ -1,0 +1,264 @@
+"""CPU oracle for the Progressive Thought Encoding decode step.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, float64 restatement of what the paper defines for one decode step
+under a fixed-size cache.  It shares no code with the CUDA path and is imported
+only by the tests, by the smoke check and by the benchmark's CPU-baseline leg.
+
+What follows which passage
+--------------------------
+* cache bookkeeping  : Sec. 3.1 (the cache grows by one entry per decoded token),
+  Sec. 3.2 (a cache policy D prunes the context at every step), Sec. 3.3 ("until
+  the KV cache is full ... earlier tokens are evicted"; sliding-window policy),
+  Sec. 4.1 implementation details (a fraction of the tokens is evicted on
+  saturation -> chunk size E).
+* attention          : the two unnumbered equations of Sec. 3.1:
+  o = softmax(q K^T / sqrt(d)) V over the cache including the new token.
+* progressive encode : Eq. (3) of Sec. 3.3 (the bracketed term named S_e), the
+  accumulation rule S_e <- Normalize(S_e + S'_e) and the bootstrap initialisation
+  from global tokens stated right after it.
+
+Readings taken where the paper is silent or garbled (each is switchable or pinned
+in the tests where the mathematics allows):
+* the third projection printed in Eq. (3) is W^a_V (the symbol list and the
+  initialisation formula use W^a_V);
+* q_g is [G, d_q]; W^a_Q is [r, d_q]; W^a_K and W^a_V are [r, d_kv]; a token's
+  evicted key/value is the concatenation of all KV heads (d_kv = H_kv * D); the
+  state S_e is [G, r] per layer per sequence;
+* Normalize: mode 0 divides each of the G rows by max(||row||_2, 1e-12), mode 1
+  divides the matrix by max(||S||_F, 1e-12), mode 2 does nothing.
+  -- parity unpinned: the paper does not define Normalize.
+* concatenated-heads vs per-head encoding -- parity unpinned (paper silent).
+* S_0 is not normalised (the initialisation formula carries no Normalize)
+  -- parity unpinned.
+* no softmax and no scaling inside the encoder (Eq. (3) has neither);
+* order inside a step: evict, append, attend; the live set never exceeds W;
+* eviction is FIFO by arrival and freed slots are reused FIFO.
+
+All arithmetic is float64.  Library primitives used as steps: numpy matmul, exp.
+"""
+from __future__ import annotations
+
+from collections import deque
+
+import numpy as np
+
+F64 = np.float64
+
+
+# ----------------------------------------------------------------------------------
+# Attention (Sec. 3.1)
+# ----------------------------------------------------------------------------------
+def attention_one_head(q, K, V):
+    """softmax(q K^T / sqrt(d)) V for one query vector.
+
+    q [D]; K, V [n, D].  Returns (o [D], lse) with lse = log sum_j exp(s_j).
+    """
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    d = q.shape[0]
+    s = (K @ q) / np.sqrt(F64(d))
+    smax = np.max(s)
+    e = np.exp(s - smax)
+    z = np.sum(e)
+    p = e / z
+    o = p @ V
+    return o, smax + np.log(z)
+
+
+def attention_gqa(q, K, V):
+    """Grouped-query decode attention of one token.
+
+    q [Hq, D]; K, V [n, Hkv, D] (the live cache entries, in any order).
+    Query head h reads KV head floor(h / (Hq/Hkv)).  Returns (o [Hq, D], lse [Hq]).
+    """
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    Hq, D = q.shape
+    Hkv = K.shape[1]
+    assert Hq % Hkv == 0
+    g = Hq // Hkv
+    o = np.zeros((Hq, D), F64)
+    lse = np.zeros((Hq,), F64)
+    for h in range(Hq):
+        o[h], lse[h] = attention_one_head(q[h], K[:, h // g, :], V[:, h // g, :])
+    return o, lse
+
+
+# ----------------------------------------------------------------------------------
+# Progressive encoder (Sec. 3.3, Eq. (3) and the two sentences after it)
+# ----------------------------------------------------------------------------------
+def normalize(S, mode=0, eps=1e-12):
+    S = np.asarray(S, F64)
+    if mode == 0:
+        n = np.sqrt(np.sum(S * S, axis=-1, keepdims=True))
+        return S / np.maximum(n, eps)
+    if mode == 1:
+        n = np.sqrt(np.sum(S * S))
+        return S / max(n, eps)
+    if mode == 2:
+        return S.copy()
+    raise ValueError("normalize mode")
+
+
+def latent_queries(Wq_a, q_g):
+    """Q_a = W^a_Q q_g for each of the G global queries: [G, r]."""
+    return np.asarray(q_g, F64) @ np.asarray(Wq_a, F64).T
+
+
+def context_state(Qa, Wk_a, Wv_a, K_e, V_e):
+    """The bracketed term of Eq. (3): ((W^a_Q q_g)(W^a_K K_e)^T)(W^a_V V_e).
+
+    Qa [G, r]; Wk_a, Wv_a [r, d_kv]; K_e, V_e [m, d_kv] (one row per evicted token).
+    Returns [G, r].
+    """
+    Ka = np.asarray(K_e, F64) @ np.asarray(Wk_a, F64).T      # [m, r]
+    Va = np.asarray(V_e, F64) @ np.asarray(Wv_a, F64).T      # [m, r]
+    P = np.asarray(Qa, F64) @ Ka.T                           # [G, m]
+    return P @ Va                                            # [G, r]
+
+
+def initial_state(Qa, Wk_a, Wv_a, k_g, v_g):
+    """Bootstrap state from the global tokens; zero when there are none (#Global-0)."""
+    if k_g is None or v_g is None:
+        return np.zeros((Qa.shape[0], np.asarray(Wv_a).shape[0]), F64)
+    return context_state(Qa, Wk_a, Wv_a, k_g, v_g)
+
+
+def encode_update(S, Qa, Wk_a, Wv_a, K_e, V_e, mode=0):
+    """S <- Normalize(S + S') with S' the context state of the evicted rows."""
+    return normalize(np.asarray(S, F64) + context_state(Qa, Wk_a, Wv_a, K_e, V_e), mode)
+
+
+# ----------------------------------------------------------------------------------
+# Cache with explicit bookkeeping (no modular index arithmetic anywhere)
+# ----------------------------------------------------------------------------------
+class _Seq:
+    """One (layer, sequence) cache: live tokens in arrival order + FIFO free slots."""
+
+    def __init__(self, W, Hkv, D):
+        self.live = deque()                 # token indices, oldest first
+        self.slot_of = {}                   # token index -> slot
+        self.free = deque(range(W))         # free slots, reused in FIFO order
+        self.K = np.zeros((W, Hkv, D), F64)
+        self.V = np.zeros((W, Hkv, D), F64)
+        self.n_appended = 0
+
+
+class OracleCache:
+    """Reference decode state for L layers x B sequences."""
+
+    def __init__(self, *, n_layers, batch, n_q_heads, n_kv_heads, head_dim, window,
+                 evict_chunk=1, n_global=32, rank=32, normalize_mode=0, encode_enabled=1):
+        assert n_q_heads % n_kv_heads == 0 and 1 <= evict_chunk <= window
+        self.L, self.B = n_layers, batch
+        self.Hq, self.Hkv, self.D = n_q_heads, n_kv_heads, head_dim
+        self.W, self.E = window, evict_chunk
+        self.G, self.r = n_global, rank
+        self.mode, self.encode_enabled = normalize_mode, encode_enabled
+        self.seqs = [[_Seq(window, n_kv_heads, head_dim) for _ in range(batch)] for _ in range(n_layers)]
+        self.enc = [None] * n_layers        # (Qa, Wk_a, Wv_a)
+        self.S = [None] * n_layers          # [B, G, r]
+        self.staged = [[None] * batch for _ in range(n_layers)]   # (K_e, V_e) of the last append
+
+    # -- set-up ------------------------------------------------------------------------
+    def set_encoder(self, layer, Wq_a, Wk_a, Wv_a, q_g, k_g=None, v_g=None):
+        Qa = latent_queries(Wq_a, q_g)
+        S0 = initial_state(Qa, Wk_a, Wv_a, k_g, v_g)
+        self.enc[layer] = (Qa, np.asarray(Wk_a, F64), np.asarray(Wv_a, F64))
+        self.S[layer] = np.repeat(S0[None], self.B, axis=0)
+
+    # -- a1: append / evict ---------------------------------------------------------------
+    def append_evict(self, layer, k_new, v_new, active=None):
+        """Token arrives for every active sequence.  Returns per-sequence records:
+        slot [B] (-1 inactive), evicted token lists, evicted slot lists."""
+        k_new = np.asarray(k_new, F64)
+        v_new = np.asarray(v_new, F64)
+        slots = np.full((self.B,), -1, np.int64)
+        ev_tokens, ev_slots = [], []
+        for b in range(self.B):
+            c = self.seqs[layer][b]
+            self.staged[layer][b] = None
+            if active is not None and not active[b]:
+                ev_tokens.append([])
+                ev_slots.append([])
+                continue
+            toks, sl = [], []
+            if len(c.live) == self.W:
+                for _ in range(self.E):
+                    t_old = c.live.popleft()
+                    s_old = c.slot_of.pop(t_old)
+                    toks.append(t_old)
+                    sl.append(s_old)
+                    c.free.append(s_old)
+                Ke = np.stack([c.K[s].reshape(-1) for s in sl])   # [m, d_kv], age order
+                Ve = np.stack([c.V[s].reshape(-1) for s in sl])
+                self.staged[layer][b] = (Ke, Ve)
+            s_new = c.free.popleft()
+            t = c.n_appended
+            c.K[s_new] = k_new[b]
+            c.V[s_new] = v_new[b]
+            c.live.append(t)
+            c.slot_of[t] = s_new
+            c.n_appended = t + 1
+            slots[b] = s_new
+            ev_tokens.append(toks)
+            ev_slots.append(sl)
+        return slots, ev_tokens, ev_slots
+
+    # -- a3: encode -----------------------------------------------------------------------
+    def encode(self, layer, K_e=None, V_e=None):
+        """Fold evicted rows into the state.  K_e/V_e: per-sequence list of [m_b, d_kv]
+        arrays (or None entries); default = the rows staged by the last append."""
+        if not self.encode_enabled:
+            return
+        if self.enc[layer] is None:        # no encoder set for this layer: nothing to fold into
+            return
+        Qa, Wk, Wv = self.enc[layer]
+        for b in range(self.B):
+            if K_e is None:
+                st = self.staged[layer][b]
+                if st is None:
+                    continue
+                Ke, Ve = st
+            else:
+                Ke, Ve = K_e[b], V_e[b]
+                if Ke is None or len(Ke) == 0:
+                    continue
+            self.S[layer][b] = encode_update(self.S[layer][b], Qa, Wk, Wv, Ke, Ve, self.mode)
+
+    # -- a2: attention -----------------------------------------------------------------------
+    def decode_attn(self, layer, q, active=None):
+        q = np.asarray(q, F64)
+        o = np.zeros((self.B, self.Hq, self.D), F64)
+        lse = np.zeros((self.B, self.Hq), F64)
+        for b in range(self.B):
+            if active is not None and not active[b]:
+                continue
+            c = self.seqs[layer][b]
+            if not c.live:
+                continue
+            sl = [c.slot_of[t] for t in c.live]
+            o[b], lse[b] = attention_gqa(q[b], c.K[sl], c.V[sl])
+        return o, lse
+
+    # -- a4: one whole step for one layer --------------------------------------------------------
+    def decode_step(self, layer, q, k_new, v_new, active=None):
+        rec = self.append_evict(layer, k_new, v_new, active)
+        self.encode(layer)
+        o, lse = self.decode_attn(layer, q, active)
+        return o, lse, rec
+
+    # -- views ---------------------------------------------------------------------------------
+    def ring(self, layer):
+        """(oldest-token slot or 0, live count, tokens appended) per sequence."""
+        head = np.zeros((self.B,), np.int64)
+        count = np.zeros((self.B,), np.int64)
+        n_app = np.zeros((self.B,), np.int64)
+        for b in range(self.B):
+            c = self.seqs[layer][b]
+            count[b] = len(c.live)
+            n_app[b] = c.n_appended
+            head[b] = c.slot_of[c.live[0]] if c.live else 0
+        return head, count, n_app
