@@ -1,0 +1,164 @@
+/*
+ * ptenc.h -- C ABI of the Progressive Thought Encoding decode hot path (sm_100a).
+ *
+ * One decode step under a fixed-size KV cache, per layer and per sequence:
+ *   a1  ring-buffer append / evict           (Sec. 3.2 cache policy D; Sec. 3.3 "until the KV
+ *                                             cache is full ... earlier tokens evicted"; Sec. 4.1
+ *                                             implementation details: a fraction of the tokens is
+ *                                             evicted on saturation)
+ *   a2  grouped-query decode attention       (Sec. 3.1, the two attention equations: the new query
+ *                                             attends over the cache including the new token)
+ *   a3  progressive encode of evicted tokens (Sec. 3.3, Eq. (3): S' = ((W^a_Q q_g)(W^a_K K_e)^T)(W^a_V V_e);
+ *                                             S <- Normalize(S + S'); bootstrap from global tokens)
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ * - Every data pointer is a DEVICE pointer unless the parameter is marked "host".
+ *   Tensors are contiguous, row-major in the index order written next to them, 16-byte aligned.
+ * - The caller owns all memory.  The library never allocates or frees device memory; its state lives
+ *   in the workspace handed to ptenc_cache_create.  The handle itself is a small host object.
+ * - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is enqueued on it and
+ *   the call returns without synchronising, except where stated.
+ * - `layer` is 0..n_layers-1, or -1 meaning "all layers in one call": every tensor argument then gains
+ *   a leading [n_layers] dimension.
+ * - `active` ([batch] bytes, may be NULL = all active) masks sequences: an inactive sequence's cache and
+ *   state are untouched and its output rows are not written.
+ * - Return value: PTENC_OK or a negative error code.  Arguments are validated on the host before any
+ *   launch; nothing is launched when an error is returned.  Device-side anomalies (a bounded wait that
+ *   ran out, an index outside its range) never trap: they set a status word read by ptenc_cache_status.
+ * - A handle may be used from one host thread and one stream at a time.
+ * - Storage dtype (ptenc_config.dtype) applies to q, k, v, out, the rings and the encoder weights;
+ *   the state S, the latent queries Q_a, lse and all accumulation are fp32.
+ */
+#ifndef PTENC_H
+#define PTENC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define PTENC_API __attribute__((visibility("default")))
+#else
+#define PTENC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PTENC_OK              0
+#define PTENC_EINVAL         -1   /* NULL pointer, value out of range, layer out of range            */
+#define PTENC_ESHAPE         -2   /* shape unsupported (heads not divisible, head_dim, G, r limits)  */
+#define PTENC_EALIGN         -3   /* a pointer is not 16-byte aligned (workspace: 1024)              */
+#define PTENC_EWORKSPACE     -4   /* workspace smaller than ptenc_workspace_bytes reports            */
+#define PTENC_ECUDA          -5   /* a CUDA runtime / driver call failed                             */
+#define PTENC_EDEVICE_STATUS -6   /* the device status word is non-zero                              */
+
+#define PTENC_DTYPE_FP32 0
+#define PTENC_DTYPE_BF16 1
+
+#define PTENC_NORM_ROW_L2    0    /* each of the G state rows divided by max(||row||_2, 1e-12)        */
+#define PTENC_NORM_FROBENIUS 1    /* whole state divided by max(||S||_F, 1e-12)                       */
+#define PTENC_NORM_NONE      2
+
+typedef struct ptenc_cache ptenc_cache;   /* opaque host handle */
+
+typedef struct {
+  int32_t n_layers;        /* L                                                                    */
+  int32_t batch;           /* B  sequences                                                          */
+  int32_t n_q_heads;       /* H_q                                                                   */
+  int32_t n_kv_heads;      /* H_kv, divides H_q                                                     */
+  int32_t head_dim;        /* D, multiple of 8, <= 256                                              */
+  int32_t window;          /* W  cache budget: tokens kept per sequence per layer                   */
+  int32_t evict_chunk;     /* E  tokens evicted when the cache is full, 1..W                        */
+  int32_t n_global;        /* G  number of state vectors (global query tokens), 1..128              */
+  int32_t rank;            /* r  length of each state vector, 1..128                                */
+  int32_t dtype;           /* PTENC_DTYPE_*                                                         */
+  int32_t normalize_mode;  /* PTENC_NORM_*                                                          */
+  int32_t encode_enabled;  /* 0: state stays at its initial value ("Global-Only" ablation, Sec. 4.3) */
+  int32_t device;          /* CUDA device ordinal the workspace lives on                            */
+  int32_t reserved[3];     /* must be zero                                                          */
+} ptenc_config;
+
+/* Bytes of device workspace a cache with this configuration needs.  Host only, launches nothing.
+ * Layout (all inside the workspace): K and V rings [L][B][H_kv][W][D]; ring state head/count (int32)
+ * and n_appended (int64) [L][B]; evicted-row staging [L][B][E][H_kv*D] for K and for V; state S
+ * [L][B][G][r] fp32; per layer Q_a [G][r] fp32 and copies of W^a_K, W^a_V; split-K partials; status. */
+PTENC_API int ptenc_workspace_bytes(const ptenc_config* cfg /*host*/, size_t* bytes /*host, out*/);
+
+/* Binds a cache to `dev_workspace` (1024-byte aligned, >= ptenc_workspace_bytes) and zeroes it on
+ * `stream`: every ring empty, every state zero, no encoder set.  The workspace must stay allocated
+ * until ptenc_cache_destroy.  Copying the workspace is a checkpoint of the whole decode state. */
+PTENC_API int ptenc_cache_create(const ptenc_config* cfg /*host*/, void* dev_workspace, size_t bytes,
+                       void* stream, ptenc_cache** out /*host, out*/);
+
+/* Frees the host handle only. */
+PTENC_API int ptenc_cache_destroy(ptenc_cache* c);
+
+/* Empties the rings of the sequences with seq_mask[b] != 0 (NULL = all) in every layer and puts their
+ * state back to the layer's initial state S_0 (zero when no encoder was set). */
+PTENC_API int ptenc_cache_reset(ptenc_cache* c, const uint8_t* seq_mask /*[B], nullable*/, void* stream);
+
+/* Encoder set-up for one layer (Sec. 3.3): stores W^a_K, W^a_V, computes Q_a = q_g W^a_Q^T [G,r] and the
+ * initial state S_0 = (Q_a (k_g W^a_K^T)^T)(v_g W^a_V^T) (the bootstrap from global tokens), and sets
+ * every sequence's state to S_0 (not normalised).  k_g == NULL or v_g == NULL gives S_0 = 0 (the
+ * "#Global-0" ablation).  Shapes: Wq_a [r, H_q*D]; Wk_a, Wv_a [r, H_kv*D]; q_g [G, H_q*D]; k_g, v_g
+ * [G, H_kv*D]; all in the storage dtype.  layer = -1 is not accepted here. */
+PTENC_API int ptenc_set_encoder(ptenc_cache* c, int layer, const void* Wq_a, const void* Wk_a, const void* Wv_a,
+                      const void* q_g, const void* k_g /*nullable*/, const void* v_g /*nullable*/,
+                      void* stream);
+
+/* a1.  For each active sequence the token with key/value k_new/v_new [B, H_kv, D] arrives.  If the
+ * sequence already holds W tokens, its E oldest tokens are evicted first (FIFO): their K/V rows are
+ * copied, oldest first and KV heads concatenated, to the staging area for ptenc_encode, and their slots
+ * are freed in that order.  The token is then stored in the oldest free slot.  With FIFO reuse the slot
+ * of the t-th token of a sequence is t mod W.  Optional outputs ([B] each, nullable): slot_out = slot
+ * written (-1 inactive); evict_first_out = index of the oldest evicted token (-1 if none);
+ * n_evicted_out = number of tokens evicted (0 or E). */
+PTENC_API int ptenc_append_evict(ptenc_cache* c, int layer, const void* k_new, const void* v_new,
+                       const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
+                       int32_t* n_evicted_out, void* stream);
+
+/* a2.  out[b,h,:] = softmax(q[b,h,:] . K_live^T / sqrt(D)) V_live over the live tokens of KV head
+ * floor(h / (H_q/H_kv)), the token appended last included.  q, out [B, H_q, D] (storage dtype);
+ * lse_out [B, H_q] fp32 (nullable) = natural-log sum of exp of the scaled scores.  Sequences with an
+ * empty cache are skipped like inactive ones. */
+PTENC_API int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* active,
+                      void* out, float* lse_out, void* stream);
+
+/* a3.  Folds evicted tokens into the state: S[b] <- Normalize(S[b] + (Q_a K_a^T) V_a) with
+ * K_a = K_e W^a_K^T, V_a = V_e W^a_V^T.  K_e, V_e [B, m_max, H_kv*D] hold n_evicted[b] <= m_max valid rows
+ * per sequence; sequences with n_evicted[b] == 0 keep their state.  K_e == NULL (then V_e, n_evicted are
+ * ignored): fold the rows staged by the last ptenc_append_evict on this layer; calling it twice folds
+ * them twice.  No-op when encode_enabled == 0 or no encoder is set for the layer. */
+PTENC_API int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e,
+                 const int32_t* n_evicted /*[B]*/, int32_t m_max, void* stream);
+
+/* a4.  One whole decode step: ptenc_append_evict ; ptenc_encode(staged rows) ; ptenc_decode_attn, with
+ * the same results as the three calls.  q, out [B, H_q, D]; k_new, v_new [B, H_kv, D] (leading [L] when
+ * layer == -1). */
+PTENC_API int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
+                      const uint8_t* active, void* out, void* stream);
+
+/* Copies one layer's ring state to device arrays [B] (each nullable): head = slot of the oldest live
+ * token, count = live tokens, n_appended = tokens ever appended. */
+PTENC_API int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* count, int64_t* n_appended,
+                   void* stream);
+
+/* Copies one layer's state to S_out [B, G, r] fp32 (device). */
+PTENC_API int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* stream);
+
+/* Synchronises the device and reads the status word into *dev_status (host).  Returns PTENC_OK when it
+ * is zero, PTENC_EDEVICE_STATUS otherwise.  The word is sticky until ptenc_cache_reset(c, NULL, ..). */
+PTENC_API int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status /*host, out, nullable*/);
+
+/* Launch statistics since creation (host counters): kernels launched by this handle. */
+PTENC_API int ptenc_launch_count(ptenc_cache* c, int64_t* n_launches /*host, out*/);
+
+/* Static string for an error code. */
+PTENC_API const char* ptenc_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PTENC_H */

@@ -1,0 +1,289 @@
+// Host side of the C ABI declared in include/ptenc.h: validation, workspace carving, launch sequencing.
+#include <new>
+#include <string.h>
+
+#include "ptenc_internal.h"
+
+namespace {
+
+constexpr size_t WS_ALIGN = 1024;
+constexpr int PART_SLOTS = 2048;      // split partial slots (two per CTA of the persistent attention grid)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  size_t K, V, head, count, n_app, stageK, stageV, n_staged, evict_first, S, S0, Qa, Wk, Wv, enc_set,
+      part_acc, part_ml, tickets, status, total;
+};
+
+int validate_config(const ptenc_config* c) {
+  if (c == nullptr) return PTENC_EINVAL;
+  if (c->n_layers <= 0 || c->batch <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 ||
+      c->window <= 0)
+    return PTENC_EINVAL;
+  if (c->evict_chunk < 1 || c->evict_chunk > c->window) return PTENC_EINVAL;
+  if (c->dtype != PTENC_DTYPE_FP32 && c->dtype != PTENC_DTYPE_BF16) return PTENC_EINVAL;
+  if (c->normalize_mode < 0 || c->normalize_mode > 2) return PTENC_EINVAL;
+  if (c->encode_enabled != 0 && c->encode_enabled != 1) return PTENC_EINVAL;
+  if (c->device < 0) return PTENC_EINVAL;
+  if (c->reserved[0] != 0 || c->reserved[1] != 0 || c->reserved[2] != 0) return PTENC_EINVAL;
+  if (c->n_q_heads % c->n_kv_heads != 0) return PTENC_ESHAPE;
+  if (c->head_dim % 8 != 0 || c->head_dim > 256) return PTENC_ESHAPE;
+  if (c->n_global < 1 || c->n_global > 128 || c->rank < 1 || c->rank > 128) return PTENC_ESHAPE;
+  if ((long long)c->n_kv_heads * c->head_dim > 8192) return PTENC_ESHAPE;
+  if ((long long)c->window > (1 << 24)) return PTENC_ESHAPE;
+  const long long rows = (long long)c->n_layers * c->batch * c->n_kv_heads * c->window;
+  if (rows >= (1ll << 31)) return PTENC_ESHAPE;
+  return PTENC_OK;
+}
+
+Layout make_layout(const ptenc_config* c) {
+  Layout o;
+  const size_t elt = c->dtype == PTENC_DTYPE_FP32 ? 4 : 2;
+  const size_t L = c->n_layers, B = c->batch, Hkv = c->n_kv_heads, D = c->head_dim, W = c->window;
+  const size_t E = c->evict_chunk, G = c->n_global, r = c->rank, d_kv = Hkv * D;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, WS_ALIGN); return at; };
+  o.K = take(L * B * Hkv * W * D * elt);
+  o.V = take(L * B * Hkv * W * D * elt);
+  o.head = take(L * B * 4);
+  o.count = take(L * B * 4);
+  o.n_app = take(L * B * 8);
+  o.stageK = take(L * B * E * d_kv * elt);
+  o.stageV = take(L * B * E * d_kv * elt);
+  o.n_staged = take(L * B * 4);
+  o.evict_first = take(L * B * 8);
+  o.S = take(L * B * G * r * 4);
+  o.S0 = take(L * G * r * 4);
+  o.Qa = take(L * G * r * 4);
+  o.Wk = take(L * r * d_kv * elt);
+  o.Wv = take(L * r * d_kv * elt);
+  o.enc_set = take(L * 4);
+  o.part_acc = take((size_t)PART_SLOTS * 8 * D * 4);
+  o.part_ml = take((size_t)PART_SLOTS * 16 * 4);
+  o.tickets = take(L * B * Hkv * 4);
+  o.status = take(64);
+  o.total = off;
+  return o;
+}
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+int check_layer(const ptenc_cache* c, int layer, int* l0, int* nl) {
+  if (c == nullptr) return PTENC_EINVAL;
+  if (layer == -1) { *l0 = 0; *nl = c->cfg.n_layers; return PTENC_OK; }
+  if (layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
+  *l0 = layer; *nl = 1;
+  return PTENC_OK;
+}
+
+cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
+                        float* lse, cudaStream_t st) {
+  if (c->fast_attn) return ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, st);
+  return ptenc_launch_attn_generic(c, l0, nl, q, active, out, lse, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int ptenc_workspace_bytes(const ptenc_config* cfg, size_t* bytes) {
+  if (bytes == nullptr) return PTENC_EINVAL;
+  int rc = validate_config(cfg);
+  if (rc != PTENC_OK) return rc;
+  *bytes = make_layout(cfg).total;
+  return PTENC_OK;
+}
+
+int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* stream, ptenc_cache** out) {
+  if (out == nullptr) return PTENC_EINVAL;
+  *out = nullptr;
+  int rc = validate_config(cfg);
+  if (rc != PTENC_OK) return rc;
+  if (ws == nullptr) return PTENC_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(ws) & (WS_ALIGN - 1)) != 0) return PTENC_EALIGN;
+  const Layout lay = make_layout(cfg);
+  if (bytes < lay.total) return PTENC_EWORKSPACE;
+
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return PTENC_ECUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return PTENC_ECUDA;
+
+  ptenc_cache* c = new (std::nothrow) ptenc_cache();
+  if (c == nullptr) return PTENC_EINVAL;
+  c->cfg = *cfg;
+  c->ws = ws;
+  c->ws_bytes = lay.total;
+  c->sm_count = prop.multiProcessorCount;
+  c->launches = 0;
+  c->fast_attn = false;
+  c->attn_grid = 0;
+
+  PtencDev& d = c->dev;
+  char* base = static_cast<char*>(ws);
+  d.L = cfg->n_layers; d.B = cfg->batch; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.D = cfg->head_dim;
+  d.W = cfg->window; d.E = cfg->evict_chunk; d.G = cfg->n_global; d.r = cfg->rank;
+  d.g = d.Hq / d.Hkv; d.d_q = d.Hq * d.D; d.d_kv = d.Hkv * d.D;
+  d.dtype = cfg->dtype; d.elt = cfg->dtype == PTENC_DTYPE_FP32 ? 4 : 2;
+  d.norm_mode = cfg->normalize_mode; d.encode_enabled = cfg->encode_enabled;
+  d.K = base + lay.K; d.V = base + lay.V;
+  d.head = reinterpret_cast<int*>(base + lay.head);
+  d.count = reinterpret_cast<int*>(base + lay.count);
+  d.n_app = reinterpret_cast<long long*>(base + lay.n_app);
+  d.stageK = base + lay.stageK; d.stageV = base + lay.stageV;
+  d.n_staged = reinterpret_cast<int*>(base + lay.n_staged);
+  d.evict_first = reinterpret_cast<long long*>(base + lay.evict_first);
+  d.S = reinterpret_cast<float*>(base + lay.S);
+  d.S0 = reinterpret_cast<float*>(base + lay.S0);
+  d.Qa = reinterpret_cast<float*>(base + lay.Qa);
+  d.Wk = base + lay.Wk; d.Wv = base + lay.Wv;
+  d.enc_set = reinterpret_cast<int*>(base + lay.enc_set);
+  d.part_acc = reinterpret_cast<float*>(base + lay.part_acc);
+  d.part_ml = reinterpret_cast<float*>(base + lay.part_ml);
+  d.tickets = reinterpret_cast<int*>(base + lay.tickets);
+  d.part_slots = PART_SLOTS;
+  d.status = reinterpret_cast<int*>(base + lay.status);
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ws, 0, lay.total, st) != cudaSuccess) { delete c; return PTENC_ECUDA; }
+
+  cudaError_t e = cudaSuccess;
+  c->fast_attn = ptenc_attn_bf16_prepare(c, &e);
+  if (e != cudaSuccess) { delete c; return PTENC_ECUDA; }
+  *out = c;
+  return PTENC_OK;
+}
+
+int ptenc_cache_destroy(ptenc_cache* c) {
+  if (c == nullptr) return PTENC_EINVAL;
+  delete c;
+  return PTENC_OK;
+}
+
+int ptenc_cache_reset(ptenc_cache* c, const uint8_t* seq_mask, void* stream) {
+  if (c == nullptr) return PTENC_EINVAL;
+  return ptenc_launch_reset(c, seq_mask, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_set_encoder(ptenc_cache* c, int layer, const void* Wq_a, const void* Wk_a, const void* Wv_a,
+                      const void* q_g, const void* k_g, const void* v_g, void* stream) {
+  if (c == nullptr || Wq_a == nullptr || Wk_a == nullptr || Wv_a == nullptr || q_g == nullptr) return PTENC_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
+  if (misaligned(Wq_a) || misaligned(Wk_a) || misaligned(Wv_a) || misaligned(q_g) || misaligned(k_g) ||
+      misaligned(v_g))
+    return PTENC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const PtencDev& d = c->dev;
+  const size_t wbytes = (size_t)d.r * d.d_kv * d.elt;
+  if (cudaMemcpyAsync(d.Wk + (size_t)layer * wbytes, Wk_a, wbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (cudaMemcpyAsync(d.Wv + (size_t)layer * wbytes, Wv_a, wbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  return ptenc_launch_set_encoder(c, layer, Wq_a, q_g, k_g, v_g, st) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_append_evict(ptenc_cache* c, int layer, const void* k_new, const void* v_new, const uint8_t* active,
+                       int32_t* slot_out, int64_t* evict_first_out, int32_t* n_evicted_out, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (k_new == nullptr || v_new == nullptr) return PTENC_EINVAL;
+  if (misaligned(k_new) || misaligned(v_new)) return PTENC_EALIGN;
+  return ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out,
+                                   static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* active, void* out, float* lse_out,
+                      void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (q == nullptr || out == nullptr) return PTENC_EINVAL;
+  if (misaligned(q) || misaligned(out)) return PTENC_EALIGN;
+  return launch_attn(c, l0, nl, q, active, out, lse_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e, const int32_t* n_evicted,
+                 int32_t m_max, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (K_e != nullptr) {
+    if (V_e == nullptr || n_evicted == nullptr || m_max < 0) return PTENC_EINVAL;
+    if (misaligned(K_e) || misaligned(V_e)) return PTENC_EALIGN;
+    if (m_max == 0) return PTENC_OK;
+  }
+  return ptenc_launch_encode(c, l0, nl, K_e, V_e, n_evicted, m_max, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
+                      const uint8_t* active, void* out, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr) return PTENC_EINVAL;
+  if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (c->cfg.encode_enabled) {
+    if (ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st) != cudaSuccess) return PTENC_ECUDA;
+  }
+  if (launch_attn(c, l0, nl, q, active, out, nullptr, st) != cudaSuccess) return PTENC_ECUDA;
+  return PTENC_OK;
+}
+
+int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* count, int64_t* n_appended, void* stream) {
+  if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t B = c->cfg.batch;
+  const PtencDev& d = c->dev;
+  if (head && cudaMemcpyAsync(head, d.head + layer * B, B * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (count && cudaMemcpyAsync(count, d.count + layer * B, B * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (n_appended &&
+      cudaMemcpyAsync(n_appended, d.n_app + layer * B, B * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  return PTENC_OK;
+}
+
+int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* stream) {
+  if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers || S_out == nullptr) return PTENC_EINVAL;
+  const PtencDev& d = c->dev;
+  const size_t n = (size_t)d.B * d.G * d.r;
+  return cudaMemcpyAsync(S_out, d.S + layer * n, n * 4, cudaMemcpyDeviceToDevice,
+                         static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status) {
+  if (c == nullptr) return PTENC_EINVAL;
+  int32_t st = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return PTENC_ECUDA;
+  if (cudaMemcpy(&st, c->dev.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PTENC_ECUDA;
+  if (dev_status) *dev_status = st;
+  return st == 0 ? PTENC_OK : PTENC_EDEVICE_STATUS;
+}
+
+int ptenc_launch_count(ptenc_cache* c, int64_t* n) {
+  if (c == nullptr || n == nullptr) return PTENC_EINVAL;
+  *n = c->launches;
+  return PTENC_OK;
+}
+
+const char* ptenc_strerror(int code) {
+  switch (code) {
+    case PTENC_OK: return "ok";
+    case PTENC_EINVAL: return "invalid argument";
+    case PTENC_ESHAPE: return "unsupported shape";
+    case PTENC_EALIGN: return "misaligned pointer";
+    case PTENC_EWORKSPACE: return "workspace too small";
+    case PTENC_ECUDA: return "CUDA call failed";
+    case PTENC_EDEVICE_STATUS: return "device status word is set";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Internal declarations shared by the translation units of libptenc (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ptenc.h"
+
+// Device status bits (sticky, OR-ed into *status).
+#define PTENC_ST_WAIT_TIMEOUT 1   // a bounded mbarrier wait ran out
+#define PTENC_ST_BAD_INDEX    2   // an index fell outside its range
+#define PTENC_ST_BAD_SCHEDULE 4   // the tile schedule did not add up
+
+// Everything a kernel needs to find the cache's buffers.  Passed by value.
+struct PtencDev {
+  int L, B, Hq, Hkv, D, W, E, G, r;
+  int g, d_q, d_kv;
+  int dtype, elt;               // storage dtype and its size in bytes
+  int norm_mode, encode_enabled;
+  char* K;                      // [L][B][Hkv][W][D]
+  char* V;
+  int* head;                    // [L][B] slot of the oldest live token
+  int* count;                   // [L][B] live tokens
+  long long* n_app;             // [L][B] tokens ever appended
+  char* stageK;                 // [L][B][E][d_kv] evicted rows of the last append, oldest first
+  char* stageV;
+  int* n_staged;                // [L][B] rows staged by the last append (0 or E)
+  long long* evict_first;       // [L][B] token index of the oldest staged row (-1 none)
+  float* S;                     // [L][B][G][r]
+  float* S0;                    // [L][G][r] initial state of the layer
+  float* Qa;                    // [L][G][r]
+  char* Wk;                     // [L][r][d_kv] storage dtype
+  char* Wv;
+  int* enc_set;                 // [L]
+  float* part_acc;              // [part_slots][8][D] split partial accumulators
+  float* part_ml;               // [part_slots][16]  (m2[8], l[8])
+  int* tickets;                 // [L][B][Hkv] arrival counters, self-cleaning
+  int part_slots;
+  int* status;
+};
+
+struct ptenc_cache {
+  ptenc_config cfg;
+  PtencDev dev;
+  size_t ws_bytes;
+  void* ws;
+  int sm_count;
+  int64_t launches;
+  bool fast_attn;               // bf16 TMA/tensor-core attention usable for this shape
+  CUtensorMap tmK, tmV;         // 2-D maps over the rings: rows = L*B*Hkv*W, cols = D
+  int attn_grid;                // persistent grid of the fast attention kernel
+};
+
+// ---- launchers (each returns a cudaError_t from the launch) -------------------------------------
+cudaError_t ptenc_launch_append_evict(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
+                                      const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
+                                      int32_t* n_evicted_out, cudaStream_t st);
+cudaError_t ptenc_launch_reset(ptenc_cache* c, const uint8_t* seq_mask, cudaStream_t st);
+cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
+                                const int32_t* n_ev, int m_max, cudaStream_t st);
+cudaError_t ptenc_launch_set_encoder(ptenc_cache* c, int layer, const void* Wq, const void* qg,
+                                     const void* kg, const void* vg, cudaStream_t st);
+cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
+                                      void* out, float* lse, cudaStream_t st);
+cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
+                                   void* out, float* lse, cudaStream_t st);
+// Host-side preparation of the fast attention path (tensor maps, attributes).  Returns false when the
+// shape is not covered, in which case the generic kernel serves it.
+bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err);
+
+// ---- small device helpers --------------------------------------------------------------------------
+__device__ __forceinline__ float ptenc_to_float(float x) { return x; }
+__device__ __forceinline__ float ptenc_to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T ptenc_from_float(float x);
+template <> __device__ __forceinline__ float ptenc_from_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 ptenc_from_float<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}

@@ -1,0 +1,209 @@
+"""GPU parity: the CUDA path through the C ABI vs the CPU oracle, same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_16839_b200 as pt
+from ptenc_inputs import CONFIGS
+
+from _harness import TOL_LSE, TOL_OUT, TOL_STATE, Pair, np64
+
+pytestmark = pytest.mark.gpu
+
+
+def _cfg(name):
+    c = dict(CONFIGS[name])
+    steps = c.pop("steps")
+    c.pop("ragged", None)
+    return c, steps
+
+
+def test_tiny_fp32_exhaustive():
+    """Configuration 1 whole: every step, sequence and head; ring state bit-exact; state within tolerance."""
+    c, steps = _cfg("tiny")
+    p = Pair(pt, seed=0, **c)
+    B = c["batch"]
+    slot = torch.empty(B, dtype=torch.int32, device="cuda")
+    first = torch.empty(B, dtype=torch.int64, device="cuda")
+    nev = torch.empty(B, dtype=torch.int32, device="cuda")
+    lse = torch.empty(B, c["n_q_heads"], dtype=torch.float32, device="cuda")
+    out = torch.empty(B, c["n_q_heads"], c["head_dim"], dtype=torch.float32, device="cuda")
+    worst = 0.0
+    for t in range(steps):
+        q = p.gen.step_q(t)
+        k, v = p.gen.step_kv(t)
+        p.cache.append_evict(0, k[0], v[0], None, slot, first, nev)
+        p.cache.encode(0)
+        p.cache.decode_attn(0, q[0], out, None, lse)
+        o_ref, lse_ref, (slots, ev_t, ev_s) = p.orc.decode_step(0, np64(q[0]), np64(k[0]), np64(v[0]))
+        assert np.array_equal(slot.cpu().numpy(), slots)
+        want_first = [e[0] if e else -1 for e in ev_t]
+        assert first.cpu().tolist() == want_first and nev.cpu().tolist() == [len(e) for e in ev_t]
+        worst = max(worst, np.abs(np64(out) - o_ref).max())
+        assert np.abs(np64(lse) - lse_ref).max() <= TOL_LSE["fp32"]
+        p.check_ring()
+        if t % 16 == 0 or t == steps - 1:
+            p.check_state()
+    assert worst <= TOL_OUT["fp32"], worst
+    assert p.cache.status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (4, 1), (7, 1), (8, 2), (14, 2), (12, 3)])
+def test_small_shapes_ragged(dtype, Hq, Hkv):
+    """Query-group sizes 1,4,7,8; window not a power of two; sequences active at random."""
+    rng = np.random.default_rng(Hq * 10 + Hkv)
+    p = Pair(pt, n_layers=2, batch=5, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=64 if dtype == "fp32" else 128,
+             window=37, evict_chunk=1, dtype=dtype, seed=3)
+    for t in range(37 * 2 + 11):
+        active = (rng.random(5) < 0.8).astype(np.uint8)
+        if t == 0:
+            active[:] = [1, 1, 0, 1, 0]
+        p.step(t, active=active)
+        if t % 9 == 0:
+            p.check_ring()
+    p.check_ring()
+    p.check_state()
+    assert p.cache.status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("W,E", [(1, 1), (2, 1), (3, 2), (5, 5), (64, 16), (100, 25), (100, 100), (130, 1), (257, 65)])
+def test_windows_and_chunks(dtype, W, E):
+    """E in {1, ceil(W/4), W}; W = 1 returns v of the newest token; ragged tile tails."""
+    p = Pair(pt, n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 32,
+             window=W, evict_chunk=E, dtype=dtype, seed=W)
+    T = min(3 * W + 5, 2 * W + 70)
+    for t in range(T):
+        p.step(t)
+        if W == 1:
+            _, v = p.gen.step_kv(t)
+            want = v[0].repeat_interleave(4, dim=1)
+            assert torch.equal(p.out[0], want)
+    p.check_ring()
+    p.check_state()
+    assert p.cache.status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_fused_step_equals_three_calls(dtype):
+    kw = dict(n_layers=3, batch=4, n_q_heads=8, n_kv_heads=2, head_dim=128, window=70, evict_chunk=3,
+              dtype=dtype, seed=5)
+    a, b, c = Pair(pt, **kw), Pair(pt, **kw), Pair(pt, **kw)
+    for t in range(160):
+        a.step(t, fused=True, all_layers=True)
+        b.step(t, fused=False, all_layers=True)
+        c.step(t, fused=True, all_layers=False)
+        assert torch.equal(a.out, b.out) and torch.equal(a.out, c.out)
+    for l in range(3):
+        assert torch.equal(a.cache.get_state(l), b.cache.get_state(l))
+        assert torch.equal(a.cache.get_state(l), c.cache.get_state(l))
+    a.check_state(); a.check_ring()
+    for x in (a, b, c):
+        x.close()
+
+
+def test_bf16_multi_tile_lse():
+    """Several 64-token tiles plus a tail, all query heads of a 7-group, lse output."""
+    p = Pair(pt, n_layers=2, batch=3, n_q_heads=28, n_kv_heads=4, head_dim=128, window=333, dtype="bf16", seed=11,
+             n_global=32, rank=32)
+    lse = torch.empty(2, 3, 28, dtype=torch.float32, device="cuda")
+    for t in range(333 + 80):
+        p.step(t)
+        if t in (0, 63, 64, 200, 332, 333, 400):
+            q = p.gen.step_q(t)
+            p.cache.decode_attn(-1, q, p.out, None, lse)
+            for l in range(2):
+                o_ref, lse_ref = p.orc.decode_attn(l, np64(q[l]))
+                assert np.abs(np64(p.out[l]) - o_ref).max() <= TOL_OUT["bf16"]
+                assert np.abs(np64(lse[l]) - lse_ref).max() <= TOL_LSE["bf16"]
+    p.check_state(); p.check_ring()
+    assert p.cache.status() == 0
+    p.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_normalize_modes_and_ablations(mode):
+    kw = dict(n_layers=1, batch=3, n_q_heads=4, n_kv_heads=2, head_dim=64, window=9, dtype="bf16", seed=mode)
+    # mode 2 never normalises: compare relative to the state's magnitude
+    p = Pair(pt, normalize_mode=mode, **kw)
+    for t in range(60):
+        p.step(t)
+    p.check_state(rel=(mode == 2))
+    p.close()
+    # Global-Only: the state never leaves S_0 (Sec. 4.3 ablation)
+    p = Pair(pt, normalize_mode=mode, encode_enabled=0, **kw)
+    s0 = p.cache.get_state(0).clone()
+    for t in range(30):
+        p.step(t)
+    assert torch.equal(p.cache.get_state(0), s0)
+    p.check_state()
+    p.close()
+    # #Global-0: zero start
+    p = Pair(pt, normalize_mode=mode, global_kv=False, **kw)
+    assert float(p.cache.get_state(0).abs().max()) == 0.0
+    for t in range(30):
+        p.step(t)
+    p.check_state(rel=(mode == 2))
+    p.close()
+
+
+def test_encode_with_caller_rows():
+    """ptenc_encode on rows supplied by the caller, ragged n_evicted, and state size independent of m."""
+    p = Pair(pt, n_layers=2, batch=4, n_q_heads=8, n_kv_heads=2, head_dim=64, window=8, dtype="bf16", seed=2,
+             n_global=16, rank=24)
+    m_max, d_kv = 11, 128
+    Ke = p.gen.generic(40, 0, (2, 4, m_max, d_kv), 1.0)
+    Ve = p.gen.generic(41, 0, (2, 4, m_max, d_kv), 1.0)
+    n_ev = torch.tensor([[0, 1, 11, 5], [3, 0, 0, 7]], dtype=torch.int32, device="cuda")
+    p.cache.encode(-1, Ke, Ve, n_ev, m_max)
+    for l in range(2):
+        rowsK = [np64(Ke[l, b, :n_ev[l, b]]) for b in range(4)]
+        rowsV = [np64(Ve[l, b, :n_ev[l, b]]) for b in range(4)]
+        p.orc.encode(l, rowsK, rowsV)
+        assert p.cache.get_state(l).shape == (4, 16, 24)
+    p.check_state()
+    # single layer call
+    p.cache.encode(1, Ke[1], Ve[1], n_ev[1], m_max)
+    p.orc.encode(1, [np64(Ke[1, b, :n_ev[1, b]]) for b in range(4)], [np64(Ve[1, b, :n_ev[1, b]]) for b in range(4)])
+    p.check_state()
+    p.close()
+
+
+def test_reset_with_mask():
+    p = Pair(pt, n_layers=2, batch=3, n_q_heads=4, n_kv_heads=1, head_dim=64, window=6, dtype="fp32", seed=8)
+    for t in range(15):
+        p.step(t)
+    mask = torch.tensor([1, 0, 1], dtype=torch.uint8, device="cuda")
+    s_before = p.cache.get_state(0).clone()
+    p.cache.reset(mask)
+    head, count, n_app = p.cache.get_ring(1)
+    assert count.tolist() == [0, 6, 0] and n_app.tolist() == [0, 15, 0]
+    s_after = p.cache.get_state(0)
+    assert torch.equal(s_after[1], s_before[1])
+    P = p.gen.encoder_params(0)
+    from oracle.ptenc_oracle import initial_state, latent_queries
+    Qa = latent_queries(np64(P["Wq_a"]), np64(P["q_g"]))
+    S0 = initial_state(Qa, np64(P["Wk_a"]), np64(P["Wv_a"]), np64(P["k_g"]), np64(P["v_g"]))
+    assert np.abs(np64(s_after[0]) - S0).max() <= 1e-4 * max(1.0, np.abs(S0).max())
+    p.close()
+
+
+def test_error_paths_on_device_box():
+    cfg = pt.make_config(n_layers=1, batch=2, n_q_heads=4, n_kv_heads=1, head_dim=64, window=8, dtype="bf16")
+    c = pt.Cache(cfg)
+    x = torch.zeros(2, 4, 64, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(2, 1, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pt.PtencError) as e:
+        c.decode_step(1, x, kv, kv, x)
+    assert e.value.code == pt.binding.PTENC_EINVAL
+    with pytest.raises(pt.PtencError) as e:
+        c.decode_step(0, x.view(-1)[1:], kv, kv, x)       # 2-byte offset: misaligned
+    assert e.value.code == pt.binding.PTENC_EALIGN
+    with pytest.raises(pt.PtencError):
+        c.decode_attn(0, None, x)
+    assert c.status() == 0
+    c.close()
