@@ -152,6 +152,12 @@ PTENC_API int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* str
  * is zero, PTENC_EDEVICE_STATUS otherwise.  The word is sticky until ptenc_cache_reset(c, NULL, ..). */
 PTENC_API int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status /*host, out, nullable*/);
 
+/* Which attention kernel serves this cache: *tensor_core_attn = 1 for the TMA + tensor-core bf16 kernel
+ * (bf16, head_dim 64 or 128, H_q/H_kv <= 8), 0 for the shape-generic kernel; *attn_grid = its persistent
+ * grid size (0 for the generic kernel).  Host only; both outputs nullable. */
+PTENC_API int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn /*host, out*/,
+                               int32_t* attn_grid /*host, out*/);
+
 /* Launch statistics since creation (host counters): kernels launched by this handle. */
 PTENC_API int ptenc_launch_count(ptenc_cache* c, int64_t* n_launches /*host, out*/);
 

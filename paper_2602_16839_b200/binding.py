@@ -21,7 +21,7 @@ NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
            "ptenc_set_encoder", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
-           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_launch_count", "ptenc_strerror"]
+           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_launch_count", "ptenc_strerror"]
 
 
 class PtencConfig(ctypes.Structure):
@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_get_ring.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ptenc_get_state.argtypes = [vp, i32, vp, vp]
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.ptenc_cache_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.ptenc_strerror.argtypes = [i32]
     lib.ptenc_strerror.restype = ctypes.c_char_p
@@ -178,6 +179,11 @@ class Cache:
         if rc not in (PTENC_OK, PTENC_EDEVICE_STATUS):
             raise PtencError(rc, "ptenc_cache_status")
         return int(st.value)
+
+    def info(self) -> dict:
+        a, b = ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(lib.ptenc_cache_info(self._h, ctypes.byref(a), ctypes.byref(b)), "ptenc_cache_info")
+        return {"tensor_core_attn": bool(a.value), "attn_grid": int(b.value)}
 
     def launch_count(self) -> int:
         n = ctypes.c_int64(0)

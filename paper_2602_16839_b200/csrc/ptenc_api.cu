@@ -1,5 +1,7 @@
 // Host side of the C ABI declared in include/ptenc.h: validation, workspace carving, launch sequencing.
 #include <new>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "ptenc_internal.h"
@@ -65,6 +67,19 @@ Layout make_layout(const ptenc_config* c) {
   o.status = take(64);
   o.total = off;
   return o;
+}
+
+// With PTENC_DEBUG set in the environment, failed CUDA calls are reported on stderr (and every launch is
+// followed by a synchronise so the report names the right step).
+bool debug_on() {
+  static int on = -1;
+  if (on < 0) { const char* e = getenv("PTENC_DEBUG"); on = (e != nullptr && e[0] != '\0' && e[0] != '0') ? 1 : 0; }
+  return on == 1;
+}
+bool ok(cudaError_t e, const char* where, cudaStream_t st = nullptr) {
+  if (e == cudaSuccess && debug_on()) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess && debug_on()) fprintf(stderr, "[ptenc] %s: %s\n", where, cudaGetErrorString(e));
+  return e == cudaSuccess;
 }
 
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
@@ -149,7 +164,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
 
   cudaError_t e = cudaSuccess;
   c->fast_attn = ptenc_attn_bf16_prepare(c, &e);
-  if (e != cudaSuccess) { delete c; return PTENC_ECUDA; }
+  if (!ok(e, "cache_create/attn_prepare")) { delete c; return PTENC_ECUDA; }
   *out = c;
   return PTENC_OK;
 }
@@ -200,8 +215,8 @@ int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* a
   if (rc != PTENC_OK) return rc;
   if (q == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(out)) return PTENC_EALIGN;
-  return launch_attn(c, l0, nl, q, active, out, lse_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
-             ? PTENC_OK : PTENC_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return ok(launch_attn(c, l0, nl, q, active, out, lse_out, st), "decode_attn", st) ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e, const int32_t* n_evicted,
@@ -226,12 +241,14 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st) != cudaSuccess)
+  if (!ok(ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st),
+          "decode_step/append_evict", st))
     return PTENC_ECUDA;
   if (c->cfg.encode_enabled) {
-    if (ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st) != cudaSuccess) return PTENC_ECUDA;
+    if (!ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step/encode", st))
+      return PTENC_ECUDA;
   }
-  if (launch_attn(c, l0, nl, q, active, out, nullptr, st) != cudaSuccess) return PTENC_ECUDA;
+  if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, st), "decode_step/attn", st)) return PTENC_ECUDA;
   return PTENC_OK;
 }
 
@@ -265,6 +282,13 @@ int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status) {
   if (cudaMemcpy(&st, c->dev.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PTENC_ECUDA;
   if (dev_status) *dev_status = st;
   return st == 0 ? PTENC_OK : PTENC_EDEVICE_STATUS;
+}
+
+int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn, int32_t* attn_grid) {
+  if (c == nullptr) return PTENC_EINVAL;
+  if (tensor_core_attn) *tensor_core_attn = c->fast_attn ? 1 : 0;
+  if (attn_grid) *attn_grid = c->fast_attn ? c->attn_grid : 0;
+  return PTENC_OK;
 }
 
 int ptenc_launch_count(ptenc_cache* c, int64_t* n) {

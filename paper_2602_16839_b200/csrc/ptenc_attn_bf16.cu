@@ -1,6 +1,613 @@
-// placeholder: fast path not built yet
+// Decode attention (step a2), bf16 fast path for sm_100a.
+//
+// Sec. 3.1: o = softmax(q K^T / sqrt(d)) V over the live cache entries (the new token included), for
+// the g = H_q / H_kv query heads that share one KV head.  The path is bound by HBM: every live K/V byte
+// is read once per step and there is no reuse between steps.
+//
+// Design
+//  * Persistent grid, one CTA per SM.  The work is the flat list of 64-token tiles of every
+//    (layer, sequence, KV head) unit that has live tokens; CTA c takes the contiguous share
+//    [c*T/n, (c+1)*T/n) of the T tiles, so no SM idles in a tail wave whatever B*H_kv is (split-K at tile
+//    granularity, sized to the machine).
+//  * A producer warp streams K and V tiles with TMA (cp.async.bulk.tensor, 128-byte swizzle, no
+//    multicast) into a ring of shared-memory stages guarded by full/empty mbarriers.
+//  * Each consumer warp owns whole tiles (tile n of the CTA goes to warp n mod NW, stage n mod STAGES; STAGES
+//    is a multiple of NW so a stage always has the same consumer warp and its full/empty barriers advance
+//    one phase per visit -- a warp can never be a phase ahead of a barrier it polls): S = Q K^T and O += P V
+//    run on warp-level bf16 mma (m16n8k16, fp32 accumulate) with the g query heads in the M rows, only to
+//    keep the FP32 pipes free; online softmax with quad shuffles; per-warp (m, l, O) partials.
+//  * Per unit the warps' partials are merged in shared memory (fp32).  A unit that is split between CTAs
+//    goes through fp32 partials in global scratch; the CTA that arrives last (atomic ticket) combines them.
+//    No CTA ever waits for another.
+//  * Every mbarrier wait is bounded; when one runs out the CTA raises a status bit, stops waiting and runs
+//    to completion on whatever is in shared memory, so barriers stay matched and nothing hangs.
+#include <math.h>
+
 #include "ptenc_internal.h"
-bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err) { *err = cudaSuccess; return false; }
-cudaError_t ptenc_launch_attn_bf16(ptenc_cache*, int, int, const void*, const uint8_t*, void*, float*, cudaStream_t) {
-  return cudaErrorNotSupported;
+
+namespace {
+
+constexpr uint32_t WAIT_POLLS = 4000000;   // bounded wait: polls before giving up (~ a second)
+
+// ------------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
+    if (mbar_test(bar, parity)) return true;
+    if (i > 128) __nanosleep(128);
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D(16x8) += A(16x16) B(16x8) with rows 8..15 of A identically zero: only c0/c1 (rows 0..7) are kept.
+__device__ __forceinline__ void mma_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  float z0, z1;
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
+      : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void consumer_sync(int nthreads) {
+  asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------ schedule
+// Live tiles of one ring: `nt` tiles starting at tile t0, cyclic over the n_t tiles of the ring.
+template <int TILE_N>
+__device__ __forceinline__ int ring_tiles(int head, int count, int W, int n_t, int* t0) {
+  *t0 = head / TILE_N;
+  if (count <= 0) return 0;
+  const int last = head + count - 1;
+  if (last < W) return last / TILE_N - *t0 + 1;
+  const int n = (n_t - *t0) + (last - W) / TILE_N + 1;
+  return n < n_t ? n : n_t;
+}
+
+struct Entry {          // one (layer, sequence) of the call
+  int head, count, nt, t0;
+};
+
+template <int D, int TILE_N, int NW, int STAGES>
+struct Smem {
+  static_assert(STAGES % NW == 0, "a stage must always be consumed by the same warp");
+  static_assert(TILE_N % 16 == 0 && (D == 64 || D == 128), "tile shape");
+  static constexpr int K_BYTES = TILE_N * D * 2;
+  static constexpr int STAGE_BYTES = 2 * K_BYTES;
+  static constexpr int Q_BYTES = 8 * D * 2;
+  static constexpr int ACC_STRIDE = D + 8;
+  static constexpr int OFF_Q = STAGES * STAGE_BYTES;
+  static constexpr int OFF_ACC = OFF_Q + 2 * Q_BYTES;
+  static constexpr int OFF_ML = OFF_ACC + NW * 8 * ACC_STRIDE * 4;
+  static constexpr int OFF_BAR = OFF_ML + NW * 16 * 4;
+  static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;
+  static constexpr int TOTAL = OFF_MISC + 64;
+};
+
+// ------------------------------------------------------------------------------------------------ kernel
+template <int D, int TILE_N, int NW, int STAGES>
+__global__ void __launch_bounds__((NW + 1) * 32, 1)
+k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+            const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
+            __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+  using SM = Smem<D, TILE_N, NW, STAGES>;
+  constexpr int NT8 = TILE_N / 8;              // 8-token n-tiles of S
+  constexpr int KT16 = TILE_N / 16;            // 16-token k-steps of P V
+  constexpr int NTHREADS = (NW + 1) * 32;
+  constexpr int NCONS = NW * 32;
+  constexpr int KSTEPS = D / 16;
+  constexpr int HALF_BYTES = TILE_N * 128;     // one 64-column half of a tile
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  float* mb_acc = reinterpret_cast<float*>(smem + SM::OFF_ACC);
+  float* mb_ml = reinterpret_cast<float*>(smem + SM::OFF_ML);
+  const uint32_t bar_full = smem_base + SM::OFF_BAR;
+  const uint32_t bar_empty = bar_full + STAGES * 8;
+  const uint32_t bar_qfull = bar_empty + STAGES * 8;
+  const uint32_t bar_qempty = bar_qfull + 2 * 8;
+  volatile int* misc = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC);
+  // misc[0] abort flag, misc[1] last-arriver flag, misc[2] start entry, misc[4..5] start prefix (int64),
+  // misc[6..7] total tiles per head-sum (int64)
+  __shared__ long long s_part[NTHREADS];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int W = p.W, B = p.B, Hkv = p.Hkv, g = p.g;
+  const int n_t = (W + TILE_N - 1) / TILE_N;
+  const int n_ent = nl * B;
+
+  // ---- set-up: barriers, zero padding rows of the Q buffers ---------------------------------------
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull + 8 * s, 1); mbar_init(bar_qempty + 8 * s, NW); }
+    misc[0] = 0; misc[1] = 0; misc[2] = -1; misc[4] = -1; misc[5] = -1;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i < 2 * SM::Q_BYTES / 4; i += NTHREADS) reinterpret_cast<uint32_t*>(smem + SM::OFF_Q)[i] = 0u;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+  // ---- schedule: total tile count and this CTA's starting entry ------------------------------------
+  auto load_entry = [&](int e) -> Entry {
+    Entry en;
+    if (e < 0 || e >= n_ent) { en.head = en.count = en.nt = en.t0 = 0; return en; }
+    const int li = e / B, b = e - li * B;
+    const size_t lb = (size_t)(l0 + li) * B + b;
+    en.head = p.head[lb];
+    en.count = (active != nullptr && active[b] == 0) ? 0 : p.count[lb];
+    if (en.head < 0 || en.head >= W || en.count < 0 || en.count > W) { en.head = 0; en.count = 0; }
+    en.nt = ring_tiles<TILE_N>(en.head, en.count, W, n_t, &en.t0);
+    return en;
+  };
+  const int chunk = (n_ent + NTHREADS - 1) / NTHREADS;
+  const int e_lo = min(tid * chunk, n_ent), e_hi = min(e_lo + chunk, n_ent);
+  long long mine = 0;
+  for (int e = e_lo; e < e_hi; ++e) mine += load_entry(e).nt;
+  s_part[tid] = mine;
+  __syncthreads();
+  long long before = 0, total = 0;
+  for (int i = 0; i < NTHREADS; ++i) {
+    const long long v = s_part[i];
+    if (i < tid) before += v;
+    total += v;
+  }
+  const long long T = total * Hkv;                     // tiles of the whole call
+  if (T == 0) return;
+  const long long n_cta = (T < (long long)gridDim.x) ? T : (long long)gridDim.x;
+  if ((long long)blockIdx.x >= n_cta) return;
+  const long long t_begin = (long long)blockIdx.x * T / n_cta;
+  const long long t_end = (long long)(blockIdx.x + 1) * T / n_cta;
+  // the thread whose chunk contains t_begin finds the entry
+  if (mine > 0 && before * Hkv <= t_begin && t_begin < (before + mine) * Hkv) {
+    long long pe = before;
+    int e = e_lo;
+    for (; e < e_hi; ++e) {
+      const int nt = load_entry(e).nt;
+      if (t_begin < (pe + nt) * Hkv) break;
+      pe += nt;
+    }
+    misc[2] = e;
+    *reinterpret_cast<volatile long long*>(&misc[4]) = pe;
+  }
+  __syncthreads();
+  const int e_start = misc[2];
+  const long long pe_start = *reinterpret_cast<volatile long long*>(&misc[4]);
+  if (e_start < 0 || e_start >= n_ent || pe_start < 0 || pe_start * Hkv > t_begin) {   // uniform over the CTA
+    if (tid == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+    return;
+  }
+
+  // Every warp walks the same sequence of units: (entry e, head h) with unit tile interval
+  // [ub, ub + nt) in the flat list, clipped to [t_begin, t_end).
+  int e = e_start;
+  Entry en = load_entry(e);
+  int h = (int)((t_begin - pe_start * Hkv) / en.nt);
+  long long ub = pe_start * Hkv + (long long)h * en.nt;
+  Entry nxt;                                             // prefetched entry e + 1
+  nxt.nt = 0; nxt.head = nxt.count = nxt.t0 = 0;
+  if (e + 1 < n_ent) nxt = load_entry(e + 1);
+
+  auto advance = [&]() {                                 // to the next unit with tiles
+    ub += en.nt;
+    if (++h < Hkv) return;
+    h = 0;
+    do {
+      ++e;
+      en = nxt;
+      if (e + 1 < n_ent) nxt = load_entry(e + 1); else nxt.nt = 0;
+    } while (e < n_ent && en.nt == 0);
+  };
+
+  const float sl2 = 1.4426950408889634f / sqrtf((float)D);
+  const uint32_t policy_dummy = 0; (void)policy_dummy;
+
+  if (warp == NW) {
+    // ================================================================ producer warp (one lane issues)
+    if (lane == 0) {
+      uint32_t n = 0;          // tiles issued by this CTA
+      uint32_t useq = 0;       // units visited
+      bool aborted = false;
+      const long long rows_total = (long long)p.L * B * Hkv * W;
+      while (ub < t_end && e < n_ent && !aborted) {
+        const long long lo = ub > t_begin ? ub : t_begin;
+        const long long hi = (ub + en.nt) < t_end ? (ub + en.nt) : t_end;
+        const int li = e / B, b = e - li * B;
+        const size_t lb = (size_t)(l0 + li) * B + b;
+        if (h < 0 || h >= Hkv || hi <= lo) { atomicOr(p.status, PTENC_ST_BAD_SCHEDULE); aborted = true; break; }
+        // Q rows of the unit
+        {
+          const uint32_t ubuf = useq & 1;
+          if (!mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) { aborted = true; break; }
+          const uint32_t qbytes = (uint32_t)(g * D * 2);
+          mbar_expect_tx(bar_qfull + 8 * ubuf, qbytes);
+          bulk_load(smem_base + SM::OFF_Q + ubuf * SM::Q_BYTES,
+                    q + (((size_t)li * B + b) * p.Hq + (size_t)h * g) * D, qbytes, bar_qfull + 8 * ubuf);
+        }
+        const long long row0 = ((long long)lb * Hkv + h) * W;
+        for (long long t = lo; t < hi; ++t, ++n) {
+          int j = en.t0 + (int)(t - ub);
+          if (j >= n_t) j -= n_t;
+          const uint32_t s = n % STAGES;
+          const long long yy = row0 + (long long)j * TILE_N;
+          if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
+            atomicOr(p.status, PTENC_ST_BAD_INDEX); aborted = true; break;
+          }
+          if (!mbar_wait(bar_empty + 8 * s, ((n / STAGES) & 1) ^ 1)) { aborted = true; break; }
+          const uint32_t dst = smem_base + s * SM::STAGE_BYTES;
+          const uint32_t fb = bar_full + 8 * s;
+          mbar_expect_tx(fb, SM::STAGE_BYTES);
+          const int y = (int)yy;
+#pragma unroll
+          for (int hf = 0; hf < D / 64; ++hf) {
+            tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
+            tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
+          }
+        }
+        ++useq;
+        advance();
+      }
+      if (aborted) {
+        atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
+        misc[0] = 1;
+        // copies still in flight must land before the CTA's shared memory goes away
+        const uint32_t back = n < (uint32_t)STAGES ? n : (uint32_t)STAGES;
+        for (uint32_t i = 0; i < back; ++i) {
+          const uint32_t nn = n - 1 - i;
+          (void)mbar_wait(bar_full + 8 * (nn % STAGES), (nn / STAGES) & 1);
+        }
+      }
+    }
+    return;
+  }
+
+  // ================================================================== consumer warps
+  const int qr = lane >> 2;          // row of the fragment = query head within the group
+  const int qc = lane & 3;
+  uint32_t n = 0;                    // CTA tile sequence number of the unit's first tile
+  uint32_t useq = 0;
+
+  while (ub < t_end && e < n_ent) {
+    const long long lo = ub > t_begin ? ub : t_begin;
+    const long long hi = (ub + en.nt) < t_end ? (ub + en.nt) : t_end;
+    const int n_mine = (int)(hi - lo);
+    const int li = e / B, b = e - li * B;
+    const int head = en.head, count = en.count;
+
+    // ---- Q fragments (A operand, rows = heads; rows >= g are zero) ------------------------------------
+    uint32_t qa[KSTEPS][2];
+    {
+      const uint32_t ubuf = useq & 1;
+      if (misc[0] == 0 && !mbar_wait(bar_qfull + 8 * ubuf, (useq >> 1) & 1)) {
+        atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
+        misc[0] = 1;
+      }
+      __syncwarp();
+      const uint8_t* qb = smem + SM::OFF_Q + ubuf * SM::Q_BYTES + qr * (D * 2) + qc * 4;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qb + ks * 32);
+        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qb + ks * 32 + 16);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_qempty + 8 * ubuf);
+    }
+
+    float m_run = -INFINITY, l_run = 0.f;
+    float o[D / 8][2];
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; }
+
+    // tiles of this unit that fall to this warp: sequence numbers n + i with (n + i) % NW == warp
+    int i0 = (int)((warp + NW - (n % NW)) % NW);
+    for (int i = i0; i < n_mine; i += NW) {
+      const uint32_t seq = n + i;
+      const uint32_t s = seq % STAGES;
+      int j = en.t0 + (int)(lo - ub) + i;
+      if (j >= n_t) j -= n_t;
+      if (misc[0] == 0 && !mbar_wait(bar_full + 8 * s, (seq / STAGES) & 1)) {
+        atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
+        misc[0] = 1;
+      }
+      __syncwarp();
+      const uint32_t kb = smem_base + s * SM::STAGE_BYTES;
+      const uint32_t vb = kb + SM::K_BYTES;
+
+      // ---- S = Q K^T (8 heads x 64 tokens), fp32 ---------------------------------------------------------
+      float sc[NT8][2];
+#pragma unroll
+      for (int nt = 0; nt < NT8; ++nt) { sc[nt][0] = 0.f; sc[nt][1] = 0.f; }
+#pragma unroll
+      for (int kp = 0; kp < KSTEPS / 2; ++kp) {
+        const int cidx = 4 * kp + (lane >> 3);               // 16-byte chunk of the row
+        const int hf = cidx >> 3, cc = cidx & 7;
+#pragma unroll
+        for (int nt = 0; nt < NT8; ++nt) {
+          const int row = 8 * nt + (lane & 7);
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(kb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), b0, b1, b2, b3);
+          mma_top(sc[nt][0], sc[nt][1], qa[2 * kp][0], qa[2 * kp][1], b0, b1);
+          mma_top(sc[nt][0], sc[nt][1], qa[2 * kp + 1][0], qa[2 * kp + 1][1], b2, b3);
+        }
+      }
+      // ---- mask slots that hold no live token -------------------------------------------------------------
+      const int slot0 = j * TILE_N;
+      int d0 = slot0 - head;
+      if (d0 < 0) d0 += W;
+      const bool full = (slot0 + TILE_N <= W) && (count == W || d0 + TILE_N <= count);
+      if (!full) {
+#pragma unroll
+        for (int nt = 0; nt < NT8; ++nt) {
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int slot = slot0 + 8 * nt + 2 * qc + x;
+            int dd = slot - head;
+            if (dd < 0) dd += W;
+            if (slot >= W || dd >= count) sc[nt][x] = -INFINITY;
+          }
+        }
+      }
+      // ---- online softmax (base 2) ---------------------------------------------------------------------------
+      float mx = sc[0][0];
+#pragma unroll
+      for (int nt = 0; nt < NT8; ++nt) { mx = fmaxf(mx, sc[nt][0]); mx = fmaxf(mx, sc[nt][1]); }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run, mx * sl2);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // all-masked row: keep exp2 arguments finite
+      const float corr = ex2(m_run - m_use);
+      float psum = 0.f;
+      uint32_t pa[KT16][2];
+#pragma unroll
+      for (int kt = 0; kt < KT16; ++kt) {
+        const float p00 = ex2(fmaf(sc[2 * kt][0], sl2, -m_use));
+        const float p01 = ex2(fmaf(sc[2 * kt][1], sl2, -m_use));
+        const float p10 = ex2(fmaf(sc[2 * kt + 1][0], sl2, -m_use));
+        const float p11 = ex2(fmaf(sc[2 * kt + 1][1], sl2, -m_use));
+        psum += (p00 + p01) + (p10 + p11);
+        pa[kt][0] = pack_bf16(p00, p01);
+        pa[kt][1] = pack_bf16(p10, p11);
+      }
+      l_run = l_run * corr + psum;
+      m_run = m_new;
+      if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+        for (int i2 = 0; i2 < D / 8; ++i2) { o[i2][0] *= corr; o[i2][1] *= corr; }
+      }
+      // ---- O += P V -------------------------------------------------------------------------------------------
+#pragma unroll
+      for (int kt = 0; kt < KT16; ++kt) {
+        const int row = 16 * kt + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int dp = 0; dp < D / 16; ++dp) {
+          const int cidx = 2 * dp + (lane >> 4);
+          const int hf = cidx >> 3, cc = cidx & 7;
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(vb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), b0, b1, b2, b3);
+          mma_top(o[2 * dp][0], o[2 * dp][1], pa[kt][0], pa[kt][1], b0, b1);
+          mma_top(o[2 * dp + 1][0], o[2 * dp + 1][1], pa[kt][0], pa[kt][1], b2, b3);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    }
+
+    // ---- merge the warps' partials of this unit ---------------------------------------------------------------
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    {
+      float* acc = mb_acc + (warp * 8 + qr) * SM::ACC_STRIDE + 2 * qc;
+#pragma unroll
+      for (int i2 = 0; i2 < D / 8; ++i2) *reinterpret_cast<float2*>(acc + 8 * i2) = make_float2(o[i2][0], o[i2][1]);
+      if (qc == 0) { mb_ml[warp * 16 + qr] = m_run; mb_ml[warp * 16 + 8 + qr] = l_run; }
+    }
+    consumer_sync(NCONS);
+
+    const long long ue = ub + en.nt;
+    const bool whole = (lo == ub) && (hi == ue);
+    const size_t unit_id = ((size_t)(l0 + li) * B + b) * Hkv + h;
+    const size_t orow0 = ((size_t)li * B + b) * p.Hq + (size_t)h * g;
+    int my_slot = 0;
+    if (!whole) my_slot = 2 * blockIdx.x + ((lo == ub) ? 1 : 0);
+    if (my_slot >= p.part_slots || h < 0 || h >= Hkv || n_mine <= 0) {      // uniform over the CTA
+      if (tid == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+      consumer_sync(NCONS);
+      n += (uint32_t)(n_mine > 0 ? n_mine : 0);
+      ++useq;
+      advance();
+      continue;
+    }
+
+    for (int idx = tid; idx < 8 * D; idx += NCONS) {
+      const int r = idx / D, d = idx - r * D;
+      float mt = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) mt = fmaxf(mt, mb_ml[w * 16 + r]);
+      float lt = 0.f, acc = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const float mw = mb_ml[w * 16 + r];
+        const float wg = (mw == -INFINITY) ? 0.f : ex2(mw - mt);
+        lt = fmaf(wg, mb_ml[w * 16 + 8 + r], lt);
+        acc = fmaf(wg, mb_acc[(w * 8 + r) * SM::ACC_STRIDE + d], acc);
+      }
+      if (whole) {
+        if (r < g) {
+          out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
+          if (lse != nullptr && d == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
+        }
+      } else {
+        p.part_acc[((size_t)my_slot * 8 + r) * D + d] = acc;
+        if (d == 0) { p.part_ml[my_slot * 16 + r] = mt; p.part_ml[my_slot * 16 + 8 + r] = lt; }
+      }
+    }
+
+    if (!whole) {
+      // ---- split unit: publish the partial; the CTA that arrives last combines ---------------------------------
+      const long long c_first = ((ub + 1) * n_cta - 1) / T;
+      const long long c_last = (ue * n_cta - 1) / T;
+      const int n_parts = (int)(c_last - c_first + 1);
+      __threadfence();
+      consumer_sync(NCONS);
+      if (tid == 0) {
+        const int old = atomicAdd(&p.tickets[unit_id], 1);
+        const int last = (old == n_parts - 1) ? 1 : 0;
+        if (last) p.tickets[unit_id] = 0;               // self-cleaning for the next launch
+        misc[1] = last;
+      }
+      consumer_sync(NCONS);
+      if (misc[1]) {
+        __threadfence();
+        for (int idx = tid; idx < 8 * D; idx += NCONS) {
+          const int r = idx / D, d = idx - r * D;
+          if (r >= g) continue;
+          float mt = -INFINITY;
+          for (long long c = c_first; c <= c_last; ++c) {
+            const int slot = 2 * (int)c + (c == c_first ? 1 : 0);
+            mt = fmaxf(mt, __ldcg(&p.part_ml[slot * 16 + r]));
+          }
+          float lt = 0.f, acc = 0.f;
+          for (long long c = c_first; c <= c_last; ++c) {
+            const int slot = 2 * (int)c + (c == c_first ? 1 : 0);
+            const float mw = __ldcg(&p.part_ml[slot * 16 + r]);
+            const float wg = (mw == -INFINITY) ? 0.f : ex2(mw - mt);
+            lt = fmaf(wg, __ldcg(&p.part_ml[slot * 16 + 8 + r]), lt);
+            acc = fmaf(wg, __ldcg(&p.part_acc[((size_t)slot * 8 + r) * D + d]), acc);
+          }
+          out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
+          if (lse != nullptr && d == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
+        }
+      }
+    }
+    consumer_sync(NCONS);       // merge buffers and misc[1] are free again
+
+    n += (uint32_t)n_mine;
+    ++useq;
+    advance();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn != nullptr) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  return fn;
+}
+
+bool make_ring_map(CUtensorMap* map, void* base, long long rows, int D, int tile_n) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)tile_n};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int NW_DEFAULT = 4;
+// 16 KiB stages, three per consumer warp.
+template <int D> struct Pick {
+  static constexpr int TILE_N = (D == 128) ? 32 : 64;
+  static constexpr int STAGES = 12;
+};
+
+template <int D>
+cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
+                     cudaStream_t st) {
+  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+  using SM = Smem<D, TN, NW, STAGES>;
+  const size_t smem = SM::TOTAL + 1024;
+  k_attn_bf16<D, TN, NW, STAGES><<<c->attn_grid, (NW + 1) * 32, smem, st>>>(
+      c->dev, c->tmK, c->tmV, l0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t prepare_t() {
+  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+  using SM = Smem<D, TN, NW, STAGES>;
+  return cudaFuncSetAttribute(k_attn_bf16<D, TN, NW, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SM::TOTAL + 1024);
+}
+
+}  // namespace
+
+bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err) {
+  *err = cudaSuccess;
+  const ptenc_config& cfg = c->cfg;
+  if (cfg.dtype != PTENC_DTYPE_BF16) return false;
+  if (cfg.head_dim != 128 && cfg.head_dim != 64) return false;
+  if (c->dev.g > 8) return false;
+  const long long rows = (long long)cfg.n_layers * cfg.batch * cfg.n_kv_heads * cfg.window;
+  const int tile_n = cfg.head_dim == 128 ? Pick<128>::TILE_N : Pick<64>::TILE_N;
+  if (!make_ring_map(&c->tmK, c->dev.K, rows, cfg.head_dim, tile_n)) return false;
+  if (!make_ring_map(&c->tmV, c->dev.V, rows, cfg.head_dim, tile_n)) return false;
+  *err = cfg.head_dim == 128 ? prepare_t<128>() : prepare_t<64>();
+  if (*err != cudaSuccess) return false;
+  c->attn_grid = c->sm_count;
+  if (2 * c->attn_grid > c->dev.part_slots) c->attn_grid = c->dev.part_slots / 2;
+  return true;
+}
+
+cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
+                                   float* lse, cudaStream_t st) {
+  if (c->cfg.head_dim == 128) return launch_t<128>(c, l0, nl, q, active, out, lse, st);
+  return launch_t<64>(c, l0, nl, q, active, out, lse, st);
 }

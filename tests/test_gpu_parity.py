@@ -207,3 +207,39 @@ def test_error_paths_on_device_box():
         c.decode_attn(0, None, x)
     assert c.status() == 0
     c.close()
+
+
+def test_tensor_core_kernel_serves_bf16_shapes():
+    """The TMA + tensor-core kernel (not the generic one) is the path taken for the paper-shaped configs."""
+    for name in ("qwen3b", "qwen7b", "llama8b"):
+        c = dict(CONFIGS[name])
+        cfg = pt.make_config(n_layers=1, batch=2, n_q_heads=c["n_q_heads"], n_kv_heads=c["n_kv_heads"],
+                             head_dim=c["head_dim"], window=128, dtype="bf16")
+        cache = pt.Cache(cfg)
+        info = cache.info()
+        assert info["tensor_core_attn"] and info["attn_grid"] >= 100
+        cache.close()
+    cache = pt.Cache(pt.make_config(n_layers=1, batch=2, n_q_heads=4, n_kv_heads=1, head_dim=64, window=64,
+                                    dtype="fp32"))
+    assert not cache.info()["tensor_core_attn"]
+    cache.close()
+
+
+def test_split_units_many_tiles_per_cta():
+    """Enough tiles that every CTA streams many pipeline rounds and most units are split between CTAs."""
+    p = Pair(pt, n_layers=2, batch=7, n_q_heads=28, n_kv_heads=4, head_dim=128, window=1500, dtype="bf16", seed=21)
+    # fill quickly: same synthetic stream on both sides, outputs checked at chosen steps only
+    for t in range(1500 + 30):
+        chk = t in (0, 1, 63, 64, 65, 700, 1499, 1500, 1501, 1529)
+        if chk:
+            p.step(t)
+        else:
+            q = p.gen.step_q(t)
+            k, v = p.gen.step_kv(t)
+            p.cache.decode_step(-1, q, k, v, p.out)
+            for l in range(2):
+                p.orc.append_evict(l, np64(k[l]), np64(v[l]))
+                p.orc.encode(l)
+    p.check_ring(); p.check_state()
+    assert p.cache.status() == 0
+    p.close()
