@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the decode hot path (append/evict + progressive encode + decode attention).
+
+One "step" = one decode step of the whole batch over all L layers, through ptenc_decode_step(layer=-1), in
+steady state: every ring full, every sequence evicting one token per step.  Workload at 1 GPU = the
+Qwen2.5-7B-shaped configuration the metric is quoted on; other workloads with --workload.
+
+    python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
+    python bench.py --impl reference ...                     (times the CPU oracle on a bounded sample)
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from ptenc_inputs import CONFIGS, make_inputs, stress_config  # noqa: E402
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0026   # (dram read + write) / algorithmic, ncu, see profiles/
+
+
+def workload_cfg(name: str) -> dict:
+    if name.startswith("stress"):
+        _, w, b = name.split("-")          # e.g. stress-w512-b16
+        c = stress_config(int(w[1:]), int(b[1:]))
+    else:
+        c = dict(CONFIGS[name])
+    c.pop("ragged", None)
+    return c
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def bytes_model(c: dict, evicting: bool = True) -> dict:
+    """Algorithmic bytes of one full-window step (all layers, all sequences active)."""
+    L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
+    elt = 2 if c["dtype"] == "bf16" else 4
+    d_q, d_kv = Hq * D, Hkv * D
+    attn = L * B * (2 * W * d_kv * elt + 2 * d_q * elt)                 # K,V window + q + o
+    append = L * B * 2 * d_kv * elt
+    enc = L * B * (2 * 1 * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) if evicting else 0
+    return {"attn": attn, "step": attn + append + enc}
+
+
+# ======================================================================================== clocks sampling
+class ClockSampler:
+    COLS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+            "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+            "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.path = f"/tmp/ptenc_clocks_{os.getpid()}.csv"
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            sel = str(device_index)
+        self.cmd = ["nvidia-smi", "-i", sel, f"--query-gpu={self.COLS}", "--format=csv,noheader,nounits", "-lms", "50"]
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(self.cmd, stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for nm, val in zip(names, parts[3:7]):
+                    if val.lower() == "active":
+                        reasons.add(nm)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            hi = [x for x in sm if x >= 0.5 * max(sm)]       # samples taken under load
+            out.update(sm_mhz=statistics.median(hi), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ======================================================================================== CPU oracle legs
+def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1):
+    """Times the CPU oracle, as it stands, on 1 layer x n_seq sequences at the full window.
+    Returns (seconds per sampled step, threads used)."""
+    from oracle.ptenc_oracle import OracleCache
+    cc = {**c, "n_layers": 1, "batch": n_seq}
+    gen = make_inputs(cc, seed=0, device="cpu")
+    orc = OracleCache(n_layers=1, batch=n_seq, n_q_heads=c["n_q_heads"], n_kv_heads=c["n_kv_heads"],
+                      head_dim=c["head_dim"], window=c["window"], evict_chunk=1, n_global=c["n_global"],
+                      rank=c["rank"])
+    P = gen.encoder_params(0)
+    orc.set_encoder(0, **{k: v.double().numpy() for k, v in P.items()})
+    pool = []
+    for t in range(4):
+        k, v = gen.step_kv(t)
+        pool.append((gen.step_q(t)[0].double().numpy(), k[0].double().numpy(), v[0].double().numpy()))
+    for t in range(c["window"]):                      # fill (not timed)
+        _, k, v = pool[t % 4]
+        orc.append_evict(0, k, v)
+    for t in range(warm):
+        orc.decode_step(0, *pool[t % 4])
+    w0, c0 = time.perf_counter(), time.process_time()
+    for t in range(n_steps):
+        orc.decode_step(0, *pool[t % 4])
+    wall = time.perf_counter() - w0
+    cpu = time.process_time() - c0
+    return wall / n_steps, max(1, int(round(cpu / wall)))
+
+
+def run_reference(args, c: dict):
+    """--impl reference: the oracle on a bounded sample; tokens/s normalised to all L layers."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_seq = 8 if c["batch"] >= 8 else c["batch"]
+    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup))
+    value = n_seq / (sec * c["n_layers"])
+    sample = (f"1 of {c['n_layers']} layers x {n_seq} of {c['batch']} sequences per step at window {c['window']} "
+              f"(full, evicting); tokens/s = {n_seq} / (step time x {c['n_layers']} layers)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * c["n_layers"] * c["batch"] / n_seq,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_block(args, c),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def config_block(args, c: dict) -> dict:
+    return {"workload": args.workload, "n_layers": c["n_layers"], "batch_per_gpu": c["batch"],
+            "n_q_heads": c["n_q_heads"], "n_kv_heads": c["n_kv_heads"], "head_dim": c["head_dim"],
+            "window": c["window"], "evict_chunk": 1, "n_global": c["n_global"], "rank": c["rank"],
+            "phase": "steady state: rings full, one eviction + encode per sequence per step",
+            "launch_mode": "all layers per call (layer = -1)",
+            "l2": "K/V rings read per step exceed the 126 MB L2 by >100x; no flush needed",
+            "parallelism": f"dp{args.gpus} (batch shards, no collective on the path)"}
+
+
+# ======================================================================================== GPU leg
+def run_gpu(args, c: dict):
+    import paper_2602_16839_b200 as pt
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
+    gen = make_inputs(c, seed=rank, device=dev)
+    cfg = pt.make_config(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=1,
+                         n_global=c["n_global"], rank=c["rank"], dtype=c["dtype"], device=local)
+    cache = pt.Cache(cfg)
+    for l in range(L):
+        P = gen.encoder_params(l)
+        cache.set_encoder(l, P["Wq_a"], P["Wk_a"], P["Wv_a"], P["q_g"], P["k_g"], P["v_g"])
+
+    # input pool: R distinct steps' worth of q/k/v, resident in HBM and mirrored in pinned host memory
+    R = 4
+    pool = []
+    for t in range(R):
+        k, v = gen.step_kv(t)
+        pool.append((gen.step_q(t), k, v))
+    out = torch.empty_like(pool[0][0])
+
+    # fill the rings (untimed): W steps reach the full window; warm-up steps then run in steady state
+    for t in range(W):
+        q, k, v = pool[t % R]
+        cache.append_evict(-1, k, v)
+    torch.cuda.synchronize()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing -----------------------------------------------------------------------
+    K, Wm = args.steps, args.warmup
+    for t in range(Wm):
+        cache.decode_step(-1, *pool[t % R], out)
+    ev_a = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    for e in ev_a + ev_b:
+        e.record()                                   # creates the CUDA handles
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    sync_all()
+    launches0 = cache.launch_count()
+    if sampler:
+        sampler.start()
+        time.sleep(0.12)
+    torch.cuda.nvtx.range_push("ptenc_timed")
+    e0.record()
+    for t in range(K):
+        cache.time_next_attn(ev_a[t], ev_b[t])
+        cache.decode_step(-1, *pool[t % R], out)
+    e1.record()
+    sync_all()
+    torch.cuda.nvtx.range_pop()
+    ms_total = e0.elapsed_time(e1)
+    launches = cache.launch_count() - launches0
+    attn_ms = [a.elapsed_time(b) for a, b in zip(ev_a, ev_b)]
+    clocks = sampler.stop() if sampler else None
+    status = cache.status()
+
+    # ---- end to end: host buffers in, host buffer out, through ptenc_decode_step_host ------------------------
+    hpool = [tuple(x.cpu().pin_memory() for x in p) for p in pool]
+    hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    staging = torch.empty(cache.host_staging_bytes(-1), dtype=torch.uint8, device=dev)
+    Ke = max(3, min(K, 100))
+    for t in range(3):
+        cache.decode_step_host(-1, *hpool[t % R], hout, staging)
+    sync_all()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for t in range(Ke):
+        cache.decode_step_host(-1, *hpool[t % R], hout, staging)
+    h1.record()
+    sync_all()
+    ms_e2e = h0.elapsed_time(h1)
+    h2d = sum(x.numel() * x.element_size() for x in hpool[0])
+    d2h = hout.numel() * hout.element_size()
+
+    # ---- max over ranks -------------------------------------------------------------------------------------
+    times = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(times[0]), float(times[1])
+
+    if rank == 0:
+        bm = bytes_model(c)
+        peak, peak_kind = measured_peak()
+        ms_step = ms_total / K
+        attn_avg_ms = sum(attn_ms) / len(attn_ms)
+        attn_gbs = bm["attn"] / (attn_avg_ms * 1e-3) / 1e9
+        step_gbs = bm["step"] / (ms_step * 1e-3) / 1e9
+        # DRAM bytes per algorithmic byte of the attention kernel, from the ncu capture summarised in
+        # profiles/attn_bf16_ncu_full_stress-w2048-b16.md (a smaller batch of the same shape; traffic grows in
+        # proportion to the tiles processed), scaled to this launch.
+        traffic = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE * bm["attn"] if c["dtype"] == "bf16" else None
+        line = {
+            "metric": METRIC, "value": world * B * K / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": c["dtype"], "data": "synthetic",
+            "config": config_block(args, c),
+            "clocks": clocks,
+            "e2e": {"value": world * B * Ke / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / Ke, "steps": Ke,
+                    "call": "ptenc_decode_step_host (pinned host q/k/v in, host out)"},
+            "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "kernel": "decode attention (k_attn_bf16)", "achieved": attn_gbs,
+                         "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
+                         "frac": attn_gbs / peak, "frac_of_8tbs": attn_gbs / NOMINAL_HBM_GBS,
+                         "traffic": traffic, "algorithmic_bytes_per_launch": bm["attn"],
+                         "avg_launch_ms": attn_avg_ms, "share_of_step": attn_avg_ms / ms_step},
+            "hbm": {"step_algorithmic_gbs": step_gbs, "frac_of_8tbs": step_gbs / NOMINAL_HBM_GBS,
+                    "frac_of_measured": step_gbs / peak, "algorithmic_bytes_per_step": bm["step"]},
+            "device_status": status,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            n_seq, n_steps = min(8, B), args.cpu_steps
+            sec, cores = oracle_sample(c, n_seq, n_steps)
+            line["cpu_baseline"] = {
+                "value": n_seq / (sec * L), "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": (f"oracle decode_step on 1 of {L} layers x {n_seq} of {B} sequences x {n_steps} steps at "
+                           f"window {W} (full, evicting); tokens/s = {n_seq} / (step time x {L} layers)")}
+        print(json.dumps(line), flush=True)
+    cache.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen7b",
+                    help="tiny | qwen3b | qwen7b | llama8b | stress-w<W>-b<B>")
+    ap.add_argument("--cpu-steps", type=int, default=128, help="steps of the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    c = workload_cfg(args.workload)
+    if args.impl == "reference":
+        run_reference(args, c)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+    run_gpu(args, c)
+
+
+if __name__ == "__main__":
+    main()

@@ -140,6 +140,17 @@ PTENC_API int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const voi
 PTENC_API int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
                       const uint8_t* active, void* out, void* stream);
 
+/* a4 with HOST buffers: the same step as ptenc_decode_step, with q, k_new, v_new, active read from host
+ * memory and out written to host memory.  The call enqueues, on `stream`, the host-to-device copies into
+ * `dev_staging` (device, 256-byte aligned, at least ptenc_host_staging_bytes), the step, and the
+ * device-to-host copy of out, and returns without synchronising: synchronise the stream before reading
+ * out_host or reusing the host inputs.  Host buffers should be page-locked for the copies to be
+ * asynchronous.  active_host may be NULL. */
+PTENC_API int ptenc_host_staging_bytes(ptenc_cache* c, int layer, size_t* bytes /*host, out*/);
+PTENC_API int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const void* k_new_host,
+                                     const void* v_new_host, const uint8_t* active_host, void* out_host,
+                                     void* dev_staging, size_t staging_bytes, void* stream);
+
 /* Copies one layer's ring state to device arrays [B] (each nullable): head = slot of the oldest live
  * token, count = live tokens, n_appended = tokens ever appended. */
 PTENC_API int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* count, int64_t* n_appended,
@@ -157,6 +168,11 @@ PTENC_API int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status /*host, out
  * grid size (0 for the generic kernel).  Host only; both outputs nullable. */
 PTENC_API int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn /*host, out*/,
                                int32_t* attn_grid /*host, out*/);
+
+/* Timing hook.  The next attention launch made through this handle (by ptenc_decode_attn, ptenc_decode_step
+ * or ptenc_decode_step_host) records the two cudaEvent_t (passed as void*) on its stream immediately
+ * before and after the attention kernel; the hook is then cleared.  NULL, NULL cancels it. */
+PTENC_API int ptenc_time_next_attn(ptenc_cache* c, void* ev_begin, void* ev_end);
 
 /* Launch statistics since creation (host counters): kernels launched by this handle. */
 PTENC_API int ptenc_launch_count(ptenc_cache* c, int64_t* n_launches /*host, out*/);

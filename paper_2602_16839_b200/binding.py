@@ -21,7 +21,8 @@ NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
            "ptenc_set_encoder", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
-           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_launch_count", "ptenc_strerror"]
+           "ptenc_host_staging_bytes", "ptenc_decode_step_host",
+           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_launch_count", "ptenc_strerror"]
 
 
 class PtencConfig(ctypes.Structure):
@@ -53,10 +54,13 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.ptenc_encode.argtypes = [vp, i32, vp, vp, vp, ctypes.c_int32, vp]
     lib.ptenc_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.ptenc_host_staging_bytes.argtypes = [vp, i32, ctypes.POINTER(u64)]
+    lib.ptenc_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u64, vp]
     lib.ptenc_get_ring.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ptenc_get_state.argtypes = [vp, i32, vp, vp]
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_cache_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+    lib.ptenc_time_next_attn.argtypes = [vp, vp, vp]
     lib.ptenc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.ptenc_strerror.argtypes = [i32]
     lib.ptenc_strerror.restype = ctypes.c_char_p
@@ -160,6 +164,17 @@ class Cache:
         _check(lib.ptenc_decode_step(self._h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(active), _ptr(out),
                                      _stream()), "ptenc_decode_step")
 
+    def host_staging_bytes(self, layer) -> int:
+        n = ctypes.c_size_t(0)
+        _check(lib.ptenc_host_staging_bytes(self._h, layer, ctypes.byref(n)), "ptenc_host_staging_bytes")
+        return int(n.value)
+
+    def decode_step_host(self, layer, q_host, k_host, v_host, out_host, dev_staging, active_host=None):
+        """Host tensors in (pinned), host tensor out; `dev_staging` is a device uint8 tensor."""
+        _check(lib.ptenc_decode_step_host(self._h, layer, _ptr(q_host), _ptr(k_host), _ptr(v_host),
+                                          _ptr(active_host), _ptr(out_host), _ptr(dev_staging),
+                                          dev_staging.numel(), _stream()), "ptenc_decode_step_host")
+
     def get_ring(self, layer):
         B = self.cfg.batch
         head = torch.empty(B, dtype=torch.int32, device=self.device)
@@ -184,6 +199,11 @@ class Cache:
         a, b = ctypes.c_int32(0), ctypes.c_int32(0)
         _check(lib.ptenc_cache_info(self._h, ctypes.byref(a), ctypes.byref(b)), "ptenc_cache_info")
         return {"tensor_core_attn": bool(a.value), "attn_grid": int(b.value)}
+
+    def time_next_attn(self, ev_begin, ev_end):
+        """ev_begin/ev_end: torch.cuda.Event(enable_timing=True) that have been recorded once (so that their
+        CUDA handles exist); they are re-recorded around the next attention kernel."""
+        _check(lib.ptenc_time_next_attn(self._h, ev_begin.cuda_event, ev_end.cuda_event), "ptenc_time_next_attn")
 
     def launch_count(self) -> int:
         n = ctypes.c_int64(0)

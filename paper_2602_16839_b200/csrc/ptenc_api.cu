@@ -94,8 +94,13 @@ int check_layer(const ptenc_cache* c, int layer, int* l0, int* nl) {
 
 cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
                         float* lse, cudaStream_t st) {
-  if (c->fast_attn) return ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, st);
-  return ptenc_launch_attn_generic(c, l0, nl, q, active, out, lse, st);
+  cudaEvent_t e0 = c->ev_attn_begin, e1 = c->ev_attn_end;
+  c->ev_attn_begin = c->ev_attn_end = nullptr;
+  if (e0 != nullptr) cudaEventRecord(e0, st);
+  cudaError_t rc = c->fast_attn ? ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, st)
+                                : ptenc_launch_attn_generic(c, l0, nl, q, active, out, lse, st);
+  if (e1 != nullptr) cudaEventRecord(e1, st);
+  return rc;
 }
 
 }  // namespace
@@ -133,6 +138,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   c->launches = 0;
   c->fast_attn = false;
   c->attn_grid = 0;
+  c->ev_attn_begin = c->ev_attn_end = nullptr;
 
   PtencDev& d = c->dev;
   char* base = static_cast<char*>(ws);
@@ -252,6 +258,60 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   return PTENC_OK;
 }
 
+namespace {
+struct HostStaging { size_t q, k, v, out, active, total, qbytes, kvbytes; };
+HostStaging host_staging(const ptenc_cache* c, int nl) {
+  HostStaging h;
+  const PtencDev& d = c->dev;
+  h.qbytes = (size_t)nl * d.B * d.d_q * d.elt;
+  h.kvbytes = (size_t)nl * d.B * d.d_kv * d.elt;
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t at = off; off = align_up(off + b, 256); return at; };
+  h.q = take(h.qbytes); h.k = take(h.kvbytes); h.v = take(h.kvbytes); h.out = take(h.qbytes);
+  h.active = take((size_t)d.B);
+  h.total = off;
+  return h;
+}
+}  // namespace
+
+int ptenc_host_staging_bytes(ptenc_cache* c, int layer, size_t* bytes) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (bytes == nullptr) return PTENC_EINVAL;
+  *bytes = host_staging(c, nl).total;
+  return PTENC_OK;
+}
+
+int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const void* k_new_host,
+                           const void* v_new_host, const uint8_t* active_host, void* out_host, void* dev_staging,
+                           size_t staging_bytes, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (q_host == nullptr || k_new_host == nullptr || v_new_host == nullptr || out_host == nullptr ||
+      dev_staging == nullptr)
+    return PTENC_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(dev_staging) & 255) != 0) return PTENC_EALIGN;
+  const HostStaging h = host_staging(c, nl);
+  if (staging_bytes < h.total) return PTENC_EWORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* sb = static_cast<char*>(dev_staging);
+  if (cudaMemcpyAsync(sb + h.q, q_host, h.qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
+  if (cudaMemcpyAsync(sb + h.k, k_new_host, h.kvbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
+  if (cudaMemcpyAsync(sb + h.v, v_new_host, h.kvbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
+  const uint8_t* act = nullptr;
+  if (active_host != nullptr) {
+    if (cudaMemcpyAsync(sb + h.active, active_host, c->cfg.batch, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return PTENC_ECUDA;
+    act = reinterpret_cast<const uint8_t*>(sb + h.active);
+  }
+  rc = ptenc_decode_step(c, layer, sb + h.q, sb + h.k, sb + h.v, act, sb + h.out, stream);
+  if (rc != PTENC_OK) return rc;
+  if (cudaMemcpyAsync(out_host, sb + h.out, h.qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PTENC_ECUDA;
+  return PTENC_OK;
+}
+
 int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* count, int64_t* n_appended, void* stream) {
   if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -288,6 +348,14 @@ int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn, int32_t* attn_gr
   if (c == nullptr) return PTENC_EINVAL;
   if (tensor_core_attn) *tensor_core_attn = c->fast_attn ? 1 : 0;
   if (attn_grid) *attn_grid = c->fast_attn ? c->attn_grid : 0;
+  return PTENC_OK;
+}
+
+int ptenc_time_next_attn(ptenc_cache* c, void* ev_begin, void* ev_end) {
+  if (c == nullptr) return PTENC_EINVAL;
+  if ((ev_begin == nullptr) != (ev_end == nullptr)) return PTENC_EINVAL;
+  c->ev_attn_begin = static_cast<cudaEvent_t>(ev_begin);
+  c->ev_attn_end = static_cast<cudaEvent_t>(ev_end);
   return PTENC_OK;
 }
 

@@ -51,6 +51,7 @@ struct ptenc_cache {
   bool fast_attn;               // bf16 TMA/tensor-core attention usable for this shape
   CUtensorMap tmK, tmV;         // 2-D maps over the rings: rows = L*B*Hkv*W, cols = D
   int attn_grid;                // persistent grid of the fast attention kernel
+  cudaEvent_t ev_attn_begin, ev_attn_end;   // one-shot timing hook around the next attention launch
 };
 
 // ---- launchers (each returns a cudaError_t from the launch) -------------------------------------
