@@ -53,6 +53,7 @@ extern "C" {
 #define PTENC_EWORKSPACE     -4   /* workspace smaller than ptenc_workspace_bytes reports            */
 #define PTENC_ECUDA          -5   /* a CUDA runtime / driver call failed                             */
 #define PTENC_EDEVICE_STATUS -6   /* the device status word is non-zero                              */
+#define PTENC_ELIMIT         -7   /* size beyond the built-in scratch of ptenc_attn_rings_static      */
 
 #define PTENC_DTYPE_FP32 0
 #define PTENC_DTYPE_BF16 1
@@ -176,6 +177,37 @@ PTENC_API int ptenc_time_next_attn(ptenc_cache* c, void* ev_begin, void* ev_end)
 
 /* Launch statistics since creation (host counters): kernels launched by this handle. */
 PTENC_API int ptenc_launch_count(ptenc_cache* c, int64_t* n_launches /*host, out*/);
+
+/* Decode attention over KV rings the caller already owns, with no workspace and no allocation of any kind.
+ * (The paper has no counterpart: this entry exists for callers, not for the method.)
+ *
+ * Who it is for: code that cannot obtain device memory at the moment it needs attention -- a serving process
+ * that committed all device memory at start-up and froze its allocator, so that a later cudaMalloc can fail or is
+ * forbidden; a latency-critical loop that must avoid the device-wide synchronisation cudaMalloc and cudaFree
+ * imply.  Such a caller cannot create a ptenc cache (it needs a workspace), so it passes its rings directly.
+ * The kernel's scratch (split-K partials, arrival tickets, a status word) lives in a 2,392,320-byte device array
+ * that is part of the library image: every GPU that loads the library holds it until the process exits.
+ *
+ * Computes exactly what ptenc_decode_attn computes with layer = -1, with the same kernel.
+ *   cfg      host; n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, dtype, device are read.  Only the
+ *            tensor-core kernel has this variant: dtype bf16, head_dim 64 or 128, n_q_heads/n_kv_heads <= 8,
+ *            else PTENC_ESHAPE.
+ *   K, V     device, [L][B][H_kv][W][D] bf16, 16-byte aligned: the rings.  Slots that hold no live token must
+ *            contain finite values (e.g. zeros).
+ *   head, count  device int32 [L][B]: slot of the oldest live token and number of live tokens of each ring;
+ *            live slots are head, head+1, ... (mod W).
+ *   q, out   device, [L][B][H_q][D] bf16; active [B] bytes or NULL; lse_out [L][B][H_q] fp32 or NULL.
+ *   status_out  device int32 or NULL: receives the kernel's status word (0 = clean) once the call has run.
+ * Limits: n_layers * batch * n_kv_heads <= 65536, else PTENC_ELIMIT (nothing is launched).
+ * The first call on a device resolves the array's device address and sets kernel attributes (once per device,
+ * with that device current); make that first call before any stream capture.  Every call on a device shares the
+ * one array, and the array keeps the previous call's contents: the entry clears the status word and the tickets on
+ * `stream` before the launch, but two calls whose kernels overlap on the GPU (different streams) race on it --
+ * serialise them.  Call it from one host thread at a time.  Asynchronous like the other entry points. */
+PTENC_API int ptenc_attn_rings_static(const ptenc_config* cfg /*host*/, const void* K, const void* V,
+                                      const int32_t* head, const int32_t* count, const void* q,
+                                      const uint8_t* active, void* out, float* lse_out, int32_t* status_out,
+                                      void* stream);
 
 /* Static string for an error code. */
 PTENC_API const char* ptenc_strerror(int code);

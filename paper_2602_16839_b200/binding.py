@@ -16,13 +16,14 @@ LIB_PATH = os.path.join(_PKG, "libptenc.so")
 
 PTENC_OK, PTENC_EINVAL, PTENC_ESHAPE, PTENC_EALIGN, PTENC_EWORKSPACE, PTENC_ECUDA, PTENC_EDEVICE_STATUS = (
     0, -1, -2, -3, -4, -5, -6)
+PTENC_ELIMIT = -7
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
            "ptenc_set_encoder", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
            "ptenc_host_staging_bytes", "ptenc_decode_step_host",
-           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_launch_count", "ptenc_strerror"]
+           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count", "ptenc_strerror"]
 
 
 class PtencConfig(ctypes.Structure):
@@ -61,6 +62,7 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_cache_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_time_next_attn.argtypes = [vp, vp, vp]
+    lib.ptenc_attn_rings_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ptenc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.ptenc_strerror.argtypes = [i32]
     lib.ptenc_strerror.restype = ctypes.c_char_p
@@ -106,6 +108,14 @@ def ptenc_workspace_bytes(cfg: PtencConfig) -> int:
     n = ctypes.c_size_t(0)
     _check(lib.ptenc_workspace_bytes(ctypes.byref(cfg), ctypes.byref(n)), "ptenc_workspace_bytes")
     return int(n.value)
+
+
+def attn_rings_static(cfg: PtencConfig, K, V, head, count, q, out, active=None, lse_out=None, status_out=None):
+    """ptenc_attn_rings_static: attention over caller-owned rings; the library allocates nothing (its scratch is a
+    device array inside the library image).  All arguments are torch CUDA tensors (or None where optional)."""
+    _check(lib.ptenc_attn_rings_static(ctypes.byref(cfg), _ptr(K), _ptr(V), _ptr(head), _ptr(count), _ptr(q),
+                                       _ptr(active), _ptr(out), _ptr(lse_out), _ptr(status_out), _stream()),
+           "ptenc_attn_rings_static")
 
 
 class Cache:

@@ -374,6 +374,7 @@ const char* ptenc_strerror(int code) {
     case PTENC_EWORKSPACE: return "workspace too small";
     case PTENC_ECUDA: return "CUDA call failed";
     case PTENC_EDEVICE_STATUS: return "device status word is set";
+    case PTENC_ELIMIT: return "size exceeds the built-in scratch limit";
     default: return "unknown error";
   }
 }

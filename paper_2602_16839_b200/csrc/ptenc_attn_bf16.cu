@@ -22,6 +22,7 @@
 //  * Every mbarrier wait is bounded; when one runs out the CTA raises a status bit, stops waiting and runs
 //    to completion on whatever is in shared memory, so barriers stay matched and nothing hangs.
 #include <math.h>
+#include <string.h>
 
 #include "ptenc_internal.h"
 
@@ -610,4 +611,132 @@ cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q
                                    float* lse, cudaStream_t st) {
   if (c->cfg.head_dim == 128) return launch_t<128>(c, l0, nl, q, active, out, lse, st);
   return launch_t<64>(c, l0, nl, q, active, out, lse, st);
+}
+
+// ================================================================================================================
+// ptenc_attn_rings_static: the same attention kernel over KV rings the caller already owns, with the kernel's
+// scratch (split partials, arrival tickets, status word) in a device array that is part of this library's image.
+// Nothing is allocated: not by this code, not through the CUDA runtime, not through torch.
+//
+// For callers that cannot allocate device memory when they want to run attention: a serving process whose
+// device memory was committed up front (rings, weights) and whose allocator is frozen, so a later cudaMalloc may
+// fail or is forbidden by policy; a latency-critical loop that must not hit the device-wide synchronisation
+// cudaMalloc / cudaFree imply.  Such a caller cannot build a ptenc workspace either, so this entry takes the rings
+// and their head/count arrays directly.
+// ================================================================================================================
+namespace {
+
+constexpr int STATIC_MAX_UNITS = 65536;                 // L * B * H_kv
+constexpr int STATIC_MAX_SLOTS = 512;                   // two per CTA of the persistent grid
+constexpr size_t STATIC_OFF_STATUS = 0;
+constexpr size_t STATIC_OFF_TICKETS = 256;
+constexpr size_t STATIC_OFF_ML = STATIC_OFF_TICKETS + (size_t)STATIC_MAX_UNITS * 4;
+constexpr size_t STATIC_OFF_ACC = STATIC_OFF_ML + (size_t)STATIC_MAX_SLOTS * 16 * 4;
+constexpr size_t STATIC_BYTES = STATIC_OFF_ACC + (size_t)STATIC_MAX_SLOTS * 8 * 128 * 4;   // 2,392,320 bytes
+
+// Lives in every GPU that loads the library, from load to exit.  In host code this name is only a stand-in for
+// the symbol, never a device address: the address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticDevice {
+  bool ready;
+  unsigned char* scratch;     // device address of g_static_scratch on that device
+  int sm_count;
+};
+StaticDevice g_static_dev[STATIC_MAX_DEVICES];
+
+// Once per device, with that device current.
+cudaError_t static_setup(int device, StaticDevice** out) {
+  if (device < 0 || device >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
+  StaticDevice& sd = g_static_dev[device];
+  if (!sd.ready) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (ptr == nullptr) return cudaErrorInvalidSymbol;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return e;
+    e = prepare_t<128>();
+    if (e != cudaSuccess) return e;
+    e = prepare_t<64>();
+    if (e != cudaSuccess) return e;
+    sd.scratch = static_cast<unsigned char*>(ptr);
+    sd.sm_count = sms;
+    sd.ready = true;
+  }
+  *out = &sd;
+  return cudaSuccess;
+}
+
+template <int D>
+cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const CUtensorMap& tmV, int grid, int nl,
+                            const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
+  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+  using SM = Smem<D, TN, NW, STAGES>;
+  k_attn_bf16<D, TN, NW, STAGES><<<grid, (NW + 1) * 32, SM::TOTAL + 1024, st>>>(
+      dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, const void* V, const int32_t* head,
+                                       const int32_t* count, const void* q, const uint8_t* active, void* out,
+                                       float* lse_out, int32_t* status_out, void* stream) {
+  if (cfg == nullptr || K == nullptr || V == nullptr || head == nullptr || count == nullptr || q == nullptr ||
+      out == nullptr)
+    return PTENC_EINVAL;
+  if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->window <= 0 ||
+      cfg->device < 0)
+    return PTENC_EINVAL;
+  if (cfg->n_q_heads % cfg->n_kv_heads != 0) return PTENC_ESHAPE;
+  if (cfg->dtype != PTENC_DTYPE_BF16 || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
+      cfg->n_q_heads / cfg->n_kv_heads > 8)
+    return PTENC_ESHAPE;                      // only the tensor-core kernel uses scratch and has this variant
+  const long long units = (long long)cfg->n_layers * cfg->batch * cfg->n_kv_heads;
+  const long long rows = units * cfg->window;
+  if (units > STATIC_MAX_UNITS || rows >= (1ll << 31)) return PTENC_ELIMIT;
+  if (((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) | reinterpret_cast<uintptr_t>(q) |
+        reinterpret_cast<uintptr_t>(out)) & 15) != 0)
+    return PTENC_EALIGN;
+
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return PTENC_ECUDA;
+  StaticDevice* sd = nullptr;
+  if (static_setup(cfg->device, &sd) != cudaSuccess) return PTENC_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  CUtensorMap tmK, tmV;
+  const int tile_n = cfg->head_dim == 128 ? Pick<128>::TILE_N : Pick<64>::TILE_N;
+  if (!make_ring_map(&tmK, const_cast<void*>(K), rows, cfg->head_dim, tile_n)) return PTENC_ECUDA;
+  if (!make_ring_map(&tmV, const_cast<void*>(V), rows, cfg->head_dim, tile_n)) return PTENC_ECUDA;
+
+  PtencDev d;
+  memset(&d, 0, sizeof(d));
+  d.L = cfg->n_layers; d.B = cfg->batch; d.Hq = cfg->n_q_heads; d.Hkv = cfg->n_kv_heads; d.D = cfg->head_dim;
+  d.W = cfg->window; d.g = d.Hq / d.Hkv; d.d_q = d.Hq * d.D; d.d_kv = d.Hkv * d.D;
+  d.dtype = PTENC_DTYPE_BF16; d.elt = 2;
+  d.K = static_cast<char*>(const_cast<void*>(K));
+  d.V = static_cast<char*>(const_cast<void*>(V));
+  d.head = const_cast<int*>(head);
+  d.count = const_cast<int*>(count);
+  d.status = reinterpret_cast<int*>(sd->scratch + STATIC_OFF_STATUS);
+  d.tickets = reinterpret_cast<int*>(sd->scratch + STATIC_OFF_TICKETS);
+  d.part_ml = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ML);
+  d.part_acc = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ACC);
+  d.part_slots = STATIC_MAX_SLOTS;
+  int grid = sd->sm_count;
+  if (2 * grid > STATIC_MAX_SLOTS) grid = STATIC_MAX_SLOTS / 2;
+
+  // The array keeps whatever the last call left: the status word and the tickets must start at zero.
+  if (cudaMemsetAsync(sd->scratch, 0, STATIC_OFF_TICKETS + (size_t)units * 4, st) != cudaSuccess) return PTENC_ECUDA;
+  cudaError_t e = cfg->head_dim == 128
+                      ? launch_static_t<128>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
+                      : launch_static_t<64>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
+  if (e != cudaSuccess) return PTENC_ECUDA;
+  if (status_out != nullptr &&
+      cudaMemcpyAsync(status_out, d.status, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  return PTENC_OK;
 }

@@ -26,7 +26,7 @@ def test_every_declared_symbol_is_exported():
 
 def test_strerror():
     assert pt.strerror(0) == "ok"
-    for code in range(-6, 0):
+    for code in range(-7, 0):
         assert pt.strerror(code) not in ("ok", "unknown error")
     assert pt.strerror(-99) == "unknown error"
 
