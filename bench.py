@@ -154,8 +154,7 @@ def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1):
 
 def run_reference(args, c: dict):
     """--impl reference: the oracle on a bounded sample; tokens/s normalised to all L layers."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if rank_env()[0] != 0:
         return
     n_seq = 8 if c["batch"] >= 8 else c["batch"]
     sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup))
@@ -184,13 +183,37 @@ def config_block(args, c: dict) -> dict:
             "parallelism": f"dp{args.gpus} (batch shards, no collective on the path)"}
 
 
+# ======================================================================================== rank plumbing
+def rank_env():
+    """(rank, world size, local rank) from the launcher's environment; (0, 1, 0) when run directly."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def shard_seed(rank: int) -> int:
+    """Each rank decodes its own batch shard: same shapes, its own synthetic stream.  Sequences are independent on
+    this path (own ring, own state), so the shards never exchange data."""
+    return int(rank)
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of per-rank timings over all ranks (the slowest rank sets the job's time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_tokens_per_s(world: int, batch_per_rank: int, steps: int, ms_total: float) -> float:
+    """Whole-job throughput: every rank decodes batch_per_rank tokens per step (weak scaling)."""
+    return world * batch_per_rank * steps / (ms_total * 1e-3)
+
+
 # ======================================================================================== GPU leg
 def run_gpu(args, c: dict):
     import paper_2602_16839_b200 as pt
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -199,7 +222,7 @@ def run_gpu(args, c: dict):
     dev = torch.device("cuda", local)
 
     L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
-    gen = make_inputs(c, seed=rank, device=dev)
+    gen = make_inputs(c, seed=shard_seed(rank), device=dev)
     cfg = pt.make_config(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=1,
                          n_global=c["n_global"], rank=c["rank"], dtype=c["dtype"], device=local)
     cache = pt.Cache(cfg)
@@ -275,10 +298,7 @@ def run_gpu(args, c: dict):
     d2h = hout.numel() * hout.element_size()
 
     # ---- max over ranks -------------------------------------------------------------------------------------
-    times = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(times[0]), float(times[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
 
     if rank == 0:
         bm = bytes_model(c)
@@ -292,12 +312,12 @@ def run_gpu(args, c: dict):
         # proportion to the tiles processed), scaled to this launch.
         traffic = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE * bm["attn"] if c["dtype"] == "bf16" else None
         line = {
-            "metric": METRIC, "value": world * B * K / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": job_tokens_per_s(world, B, K, ms_total), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": c["dtype"], "data": "synthetic",
             "config": config_block(args, c),
             "clocks": clocks,
-            "e2e": {"value": world * B * Ke / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": job_tokens_per_s(world, B, Ke, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / Ke, "steps": Ke,
                     "call": "ptenc_decode_step_host (pinned host q/k/v in, host out)"},
             "gpu_launches": launches,
