@@ -26,6 +26,23 @@
 
 #include "ptenc_internal.h"
 
+// Compile-time tunables of the D = 128 kernel (defaults: 32-token tiles = 16 KiB stages, three per consumer warp).
+#ifndef PTENC_ATTN_TILE_N_128
+#define PTENC_ATTN_TILE_N_128 32
+#endif
+#ifndef PTENC_ATTN_STAGES_128
+#define PTENC_ATTN_STAGES_128 12
+#endif
+#ifndef PTENC_ATTN_NW
+#define PTENC_ATTN_NW 4
+#endif
+#ifndef PTENC_ATTN_CTAS_PER_SM
+#define PTENC_ATTN_CTAS_PER_SM 1
+#endif
+#ifndef PTENC_ATTN_L2PROMO
+#define PTENC_ATTN_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
+
 namespace {
 
 constexpr uint32_t WAIT_POLLS = 4000000;   // bounded wait: polls before giving up (~ a second)
@@ -132,7 +149,7 @@ struct Smem {
 
 // ------------------------------------------------------------------------------------------------ kernel
 template <int D, int TILE_N, int NW, int STAGES>
-__global__ void __launch_bounds__((NW + 1) * 32, 1)
+__global__ void __launch_bounds__((NW + 1) * 32, PTENC_ATTN_CTAS_PER_SM)
 k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
             __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
@@ -557,15 +574,14 @@ bool make_ring_map(CUtensorMap* map, void* base, long long rows, int D, int tile
   cuuint32_t box[2] = {64, (cuuint32_t)tile_n};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_SWIZZLE_128B, PTENC_ATTN_L2PROMO,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int NW_DEFAULT = 4;
-// 16 KiB stages, three per consumer warp.
+constexpr int NW_DEFAULT = PTENC_ATTN_NW;
 template <int D> struct Pick {
-  static constexpr int TILE_N = (D == 128) ? 32 : 64;
-  static constexpr int STAGES = 12;
+  static constexpr int TILE_N = (D == 128) ? PTENC_ATTN_TILE_N_128 : 64;
+  static constexpr int STAGES = (D == 128) ? PTENC_ATTN_STAGES_128 : 12 / NW_DEFAULT * NW_DEFAULT;
 };
 
 template <int D>
@@ -602,7 +618,7 @@ bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err) {
   if (!make_ring_map(&c->tmV, c->dev.V, rows, cfg.head_dim, tile_n)) return false;
   *err = cfg.head_dim == 128 ? prepare_t<128>() : prepare_t<64>();
   if (*err != cudaSuccess) return false;
-  c->attn_grid = c->sm_count;
+  c->attn_grid = c->sm_count * PTENC_ATTN_CTAS_PER_SM;
   if (2 * c->attn_grid > c->dev.part_slots) c->attn_grid = c->dev.part_slots / 2;
   return true;
 }
@@ -726,7 +742,7 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   d.part_ml = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ML);
   d.part_acc = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ACC);
   d.part_slots = STATIC_MAX_SLOTS;
-  int grid = sd->sm_count;
+  int grid = sd->sm_count * PTENC_ATTN_CTAS_PER_SM;
   if (2 * grid > STATIC_MAX_SLOTS) grid = STATIC_MAX_SLOTS / 2;
 
   // The array keeps whatever the last call left: the status word and the tickets must start at zero.
