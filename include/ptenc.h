@@ -164,11 +164,13 @@ PTENC_API int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* str
  * is zero, PTENC_EDEVICE_STATUS otherwise.  The word is sticky until ptenc_cache_reset(c, NULL, ..). */
 PTENC_API int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status /*host, out, nullable*/);
 
-/* Which attention kernel serves this cache: *tensor_core_attn = 1 for the TMA + tensor-core bf16 kernel
+/* Which kernels serve this cache: *tensor_core_attn = 1 for the TMA + tensor-core bf16 attention kernel
  * (bf16, head_dim 64 or 128, H_q/H_kv <= 8), 0 for the shape-generic kernel; *attn_grid = its persistent
- * grid size (0 for the generic kernel).  Host only; both outputs nullable. */
+ * grid size (0 for the generic kernel); *tensor_core_encode = 1 when chunks of evicted tokens (E >= 2, or
+ * ptenc_encode with m_max >= 2) are folded by the tcgen05 kernel (bf16, rank 16/32/64, H_kv*D a multiple of 64),
+ * 0 when the shape-generic encoder serves them.  Host only; every output nullable. */
 PTENC_API int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn /*host, out*/,
-                               int32_t* attn_grid /*host, out*/);
+                               int32_t* attn_grid /*host, out*/, int32_t* tensor_core_encode /*host, out*/);
 
 /* Timing hook.  The next attention launch made through this handle (by ptenc_decode_attn, ptenc_decode_step
  * or ptenc_decode_step_host) records the two cudaEvent_t (passed as void*) on its stream immediately

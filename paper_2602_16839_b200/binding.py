@@ -60,7 +60,7 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_get_ring.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ptenc_get_state.argtypes = [vp, i32, vp, vp]
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
-    lib.ptenc_cache_info.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+    lib.ptenc_cache_info.argtypes = [vp] + [ctypes.POINTER(ctypes.c_int32)] * 3
     lib.ptenc_time_next_attn.argtypes = [vp, vp, vp]
     lib.ptenc_attn_rings_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ptenc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
@@ -206,9 +206,9 @@ class Cache:
         return int(st.value)
 
     def info(self) -> dict:
-        a, b = ctypes.c_int32(0), ctypes.c_int32(0)
-        _check(lib.ptenc_cache_info(self._h, ctypes.byref(a), ctypes.byref(b)), "ptenc_cache_info")
-        return {"tensor_core_attn": bool(a.value), "attn_grid": int(b.value)}
+        a, b, e = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(lib.ptenc_cache_info(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(e)), "ptenc_cache_info")
+        return {"tensor_core_attn": bool(a.value), "attn_grid": int(b.value), "tensor_core_encode": bool(e.value)}
 
     def time_next_attn(self, ev_begin, ev_end):
         """ev_begin/ev_end: torch.cuda.Event(enable_timing=True) that have been recorded once (so that their

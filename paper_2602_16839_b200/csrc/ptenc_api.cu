@@ -137,6 +137,8 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   c->sm_count = prop.multiProcessorCount;
   c->launches = 0;
   c->fast_attn = false;
+  c->tc_encode = false;
+  c->tc_stage_box = 0;
   c->attn_grid = 0;
   c->ev_attn_begin = c->ev_attn_end = nullptr;
 
@@ -171,6 +173,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   cudaError_t e = cudaSuccess;
   c->fast_attn = ptenc_attn_bf16_prepare(c, &e);
   if (!ok(e, "cache_create/attn_prepare")) { delete c; return PTENC_ECUDA; }
+  (void)ptenc_encode_tc_prepare(c);
   *out = c;
   return PTENC_OK;
 }
@@ -344,10 +347,11 @@ int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status) {
   return st == 0 ? PTENC_OK : PTENC_EDEVICE_STATUS;
 }
 
-int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn, int32_t* attn_grid) {
+int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn, int32_t* attn_grid, int32_t* tensor_core_encode) {
   if (c == nullptr) return PTENC_EINVAL;
   if (tensor_core_attn) *tensor_core_attn = c->fast_attn ? 1 : 0;
   if (attn_grid) *attn_grid = c->fast_attn ? c->attn_grid : 0;
+  if (tensor_core_encode) *tensor_core_encode = c->tc_encode ? 1 : 0;
   return PTENC_OK;
 }
 

@@ -408,6 +408,10 @@ cudaError_t launch_encode_step(ptenc_cache* c, int l0, int nl, const void* Ke, c
 cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
                                 const int32_t* n_ev, int m_max, cudaStream_t st) {
   if (encode_step_usable(c, Ke, m_max)) return launch_encode_step(c, l0, nl, Ke, Ve, n_ev, m_max, st);
+  // chunks of evicted tokens: the projections are dense contractions -> tensor cores
+  if (c->tc_encode && (Ke == nullptr ? c->dev.E : m_max) >= 2 &&
+      (Ke == nullptr || (long long)nl * c->cfg.batch * m_max >= 128))
+    return ptenc_launch_encode_tc(c, l0, nl, Ke, Ve, n_ev, m_max, st);
   if (c->cfg.dtype == PTENC_DTYPE_FP32) return launch_encode_t<float>(c, l0, nl, Ke, Ve, n_ev, m_max, 0, st);
   return launch_encode_t<__nv_bfloat16>(c, l0, nl, Ke, Ve, n_ev, m_max, 0, st);
 }

@@ -52,6 +52,10 @@ struct ptenc_cache {
   CUtensorMap tmK, tmV;         // 2-D maps over the rings: rows = L*B*Hkv*W, cols = D
   int attn_grid;                // persistent grid of the fast attention kernel
   cudaEvent_t ev_attn_begin, ev_attn_end;   // one-shot timing hook around the next attention launch
+  bool tc_encode;               // tensor-core chunk encoder usable for this shape
+  CUtensorMap tmWk, tmWv;       // 2-D maps over the encoder weights: rows = L*r, cols = d_kv
+  CUtensorMap tmStageK, tmStageV;   // 2-D maps over the staged evicted rows: rows = L*B*E, cols = d_kv
+  int tc_stage_box;             // token rows per TMA box of the staged maps
 };
 
 // ---- launchers (each returns a cudaError_t from the launch) -------------------------------------
@@ -67,6 +71,10 @@ cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void
                                       void* out, float* lse, cudaStream_t st);
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
                                    void* out, float* lse, cudaStream_t st);
+// Chunk encoder on tcgen05 (bf16, rank 16/32/64, d_kv % 64 == 0): tensor maps at create time, launch per call.
+bool ptenc_encode_tc_prepare(ptenc_cache* c);
+cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
+                                   const int32_t* n_ev, int m_max, cudaStream_t st);
 // Host-side preparation of the fast attention path (tensor maps, attributes).  Returns false when the
 // shape is not covered, in which case the generic kernel serves it.
 bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err);

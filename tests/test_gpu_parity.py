@@ -243,3 +243,51 @@ def test_split_units_many_tiles_per_cta():
     p.check_ring(); p.check_state()
     assert p.cache.status() == 0
     p.close()
+
+
+@pytest.mark.parametrize("W,E,G,r,Hkv", [(64, 16, 32, 32, 2), (600, 150, 32, 32, 4), (256, 128, 16, 16, 2),
+                                         (300, 129, 48, 64, 2), (40, 5, 8, 32, 1), (2048, 512, 32, 32, 4)])
+def test_chunk_eviction_on_the_tensor_core_encoder(W, E, G, r, Hkv):
+    """Chunks of E tokens leave at once (Sec. 4.1: 25 % of the window in the paper's runs): the projections run on
+    tcgen05; tiles of 128 tokens with ragged tails, every supported rank, state against the float64 oracle."""
+    p = Pair(pt, n_layers=2, batch=3, n_q_heads=2 * Hkv, n_kv_heads=Hkv, head_dim=128, window=W, evict_chunk=E,
+             dtype="bf16", seed=W + E, n_global=G, rank=r)
+    assert p.cache.info()["tensor_core_encode"]
+    T = W + 2 * E + 3
+    checks = {0, W - 1, W, W + 1, W + E - 1, W + E, W + E + 1, T - 1}
+    states_at = {W, W + E, T - 1}
+    for t in range(T):
+        if t in checks:
+            p.step(t)
+        else:
+            q = p.gen.step_q(t)
+            k, v = p.gen.step_kv(t)
+            p.cache.decode_step(-1, q, k, v, p.out)
+            for l in range(p.L):
+                p.orc.append_evict(l, np64(k[l]), np64(v[l]))
+                p.orc.encode(l)
+        if t in states_at:
+            p.check_state()
+            p.check_ring()
+    assert p.cache.status() == 0
+    p.close()
+
+
+def test_tensor_core_encoder_with_caller_rows_and_modes():
+    """ptenc_encode on caller-supplied chunks: ragged row counts around the 128-row tile, all three Normalize modes."""
+    for mode in (0, 1, 2):
+        p = Pair(pt, n_layers=2, batch=6, n_q_heads=8, n_kv_heads=4, head_dim=64, window=16, evict_chunk=4,
+                 dtype="bf16", seed=40 + mode, n_global=24, rank=32, normalize_mode=mode)
+        assert p.cache.info()["tensor_core_encode"]
+        m_max, d_kv = 200, 256
+        Ke = p.gen.generic(40, 0, (2, 6, m_max, d_kv), 1.0)
+        Ve = p.gen.generic(41, 0, (2, 6, m_max, d_kv), 1.0)
+        n_ev = torch.tensor([[0, 1, 127, 128, 129, 200], [200, 64, 0, 7, 130, 255]], dtype=torch.int32, device="cuda")
+        for rep in range(2):
+            p.cache.encode(-1, Ke, Ve, n_ev, m_max)
+            for l in range(2):
+                cnt = [min(int(n_ev[l, b]), m_max) for b in range(6)]
+                p.orc.encode(l, [np64(Ke[l, b, :cnt[b]]) for b in range(6)], [np64(Ve[l, b, :cnt[b]]) for b in range(6)])
+            p.check_state(rel=(mode == 2), tol=2e-4 if mode == 2 else TOL_STATE)
+        assert p.cache.status() == 0
+        p.close()
