@@ -250,12 +250,19 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!ok(ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st),
-          "decode_step/append_evict", st))
-    return PTENC_ECUDA;
-  if (c->cfg.encode_enabled) {
-    if (!ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step/encode", st))
+  if (c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0)) {
+    // ring-per-step mode: append/evict and the encode of the evicted row in one kernel
+    if (!ok(ptenc_launch_step_e1(c, l0, nl, true, k_new, v_new, active, nullptr, nullptr, nullptr, 0, st),
+            "decode_step/append_evict+encode", st))
       return PTENC_ECUDA;
+  } else {
+    if (!ok(ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st),
+            "decode_step/append_evict", st))
+      return PTENC_ECUDA;
+    if (c->cfg.encode_enabled) {
+      if (!ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step/encode", st))
+        return PTENC_ECUDA;
+    }
   }
   if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, st), "decode_step/attn", st)) return PTENC_ECUDA;
   return PTENC_OK;

@@ -167,179 +167,6 @@ k_encode_rows(PtencDev p, int l0, const T* __restrict__ Ke, const T* __restrict_
   }
 }
 
-// ---------------------------------------------------------------------------------------------------------------
-// One evicted token per sequence (E = 1, the ring-per-step mode), bf16 storage: the projections of a block of 16
-// sequences of one layer are one small matrix product X [16, d_kv] x W^T [d_kv, r] per map, done with warp-level
-// bf16 mma (fp32 accumulate) so that the layer's weights are read once per 16 sequences instead of once per
-// sequence.  Each lane fetches 8 consecutive k-values of its A row (shared memory) and of its B row (W^a, from L2)
-// with one 16-byte load and feeds them to two mma steps; the contraction index is permuted the same way on both
-// operands, which leaves the sum unchanged.  Then p = Q_a k_a, S + p v_a^T, Normalize, all in fp32.
-// ---------------------------------------------------------------------------------------------------------------
-constexpr int ES_SEQ = 16;
-constexpr int ES_THREADS = 256;
-constexpr int ES_WARPS = ES_THREADS / 32;
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__host__ __device__ inline size_t encode_step_smem(int G, int r, int d_kv) {
-  const size_t xstride = (size_t)d_kv * 2 + 64;
-  return 2 * ES_SEQ * xstride + sizeof(float) * ((size_t)ES_SEQ * 2 * r + (size_t)G * (r + 1) + (size_t)ES_SEQ * G) +
-         ES_SEQ * sizeof(int);
-}
-
-__global__ void __launch_bounds__(ES_THREADS)
-k_encode_step_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ Ke, const __nv_bfloat16* __restrict__ Ve,
-                  const int32_t* __restrict__ n_ev, int m_max) {
-  extern __shared__ __align__(16) uint8_t es_smem[];
-  const int G = p.G, r = p.r, d_kv = p.d_kv, B = p.B;
-  const int xstride = d_kv * 2 + 64;                 // bytes; = 64 mod 128 keeps the 16-byte A loads conflict-free
-  uint8_t* xk = es_smem;
-  uint8_t* xv = xk + ES_SEQ * xstride;
-  float* kv_a = reinterpret_cast<float*>(xv + ES_SEQ * xstride);   // [16][2r]: k_a | v_a of each sequence
-  float* qa = kv_a + ES_SEQ * 2 * r;                               // [G][r + 1]
-  float* pg = qa + G * (r + 1);                                    // [16][G]
-  int* has = reinterpret_cast<int*>(pg + ES_SEQ * G);              // [16]
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int nblk = (B + ES_SEQ - 1) / ES_SEQ;
-  const int li = blockIdx.x / nblk;
-  const int b0 = (blockIdx.x - li * nblk) * ES_SEQ;
-  const int l = l0 + li;
-  if (!p.encode_enabled || !p.enc_set[l]) return;
-
-  int mine = 0;
-  if (tid < ES_SEQ) {
-    const int b = b0 + tid;
-    if (b < B) mine = (Ke == nullptr) ? p.n_staged[(size_t)l * B + b] : min(n_ev[(size_t)li * B + b], m_max);
-    has[tid] = mine > 0 ? 1 : 0;
-  }
-  if (__syncthreads_or(mine > 0) == 0) return;
-
-  // ---- the evicted rows of the 16 sequences (zero rows where nothing was evicted) -----------------------------------
-  const int vpr = d_kv >> 3;                         // 16-byte vectors per row
-  for (int idx = tid; idx < ES_SEQ * vpr; idx += ES_THREADS) {
-    const int row = idx / vpr, v = idx - row * vpr;
-    uint4 k4 = make_uint4(0u, 0u, 0u, 0u), v4 = k4;
-    if (has[row]) {
-      const int b = b0 + row;
-      const size_t src = (Ke == nullptr) ? ((size_t)l * B + b) * p.E * d_kv : ((size_t)li * B + b) * m_max * d_kv;
-      const __nv_bfloat16* rk = (Ke == nullptr) ? reinterpret_cast<const __nv_bfloat16*>(p.stageK) : Ke;
-      const __nv_bfloat16* rv = (Ke == nullptr) ? reinterpret_cast<const __nv_bfloat16*>(p.stageV) : Ve;
-      k4 = *reinterpret_cast<const uint4*>(rk + src + (size_t)v * 8);
-      v4 = *reinterpret_cast<const uint4*>(rv + src + (size_t)v * 8);
-    }
-    *reinterpret_cast<uint4*>(xk + row * xstride + v * 16) = k4;
-    *reinterpret_cast<uint4*>(xv + row * xstride + v * 16) = v4;
-  }
-  const int gr = G * r;
-  for (int i = tid; i < gr; i += ES_THREADS) {
-    const int gi = i / r;
-    qa[gi * (r + 1) + (i - gi * r)] = p.Qa[(size_t)l * gr + i];
-  }
-  __syncthreads();
-
-  // ---- k_a = X_k W^a_K^T, v_a = X_v W^a_V^T : 2r/8 column tiles of 8, spread over the warps ------------------------
-  {
-    const __nv_bfloat16* Wk = reinterpret_cast<const __nv_bfloat16*>(p.Wk) + (size_t)l * r * d_kv;
-    const __nv_bfloat16* Wv = reinterpret_cast<const __nv_bfloat16*>(p.Wv) + (size_t)l * r * d_kv;
-    const int tiles_per_map = r >> 3;
-    const int n_pairs = d_kv >> 5;                   // 32 k-values per pair of mma steps
-    const int qrow = lane >> 2, qcol = lane & 3;
-    for (int tile = warp; tile < 2 * tiles_per_map; tile += ES_WARPS) {
-      const int mat = tile >= tiles_per_map ? 1 : 0;
-      const int j0 = (tile - mat * tiles_per_map) * 8;
-      const __nv_bfloat16* wrow = (mat ? Wv : Wk) + (size_t)(j0 + qrow) * d_kv + qcol * 8;
-      const uint8_t* xa = (mat ? xv : xk) + qrow * xstride + qcol * 16;
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int s0 = 0; s0 < n_pairs; s0 += 8) {
-        uint4 bw[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-          if (s0 + u < n_pairs) bw[u] = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(s0 + u) * 32));
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (s0 + u < n_pairs) {
-            const uint4 lo = *reinterpret_cast<const uint4*>(xa + (s0 + u) * 64);
-            const uint4 hi = *reinterpret_cast<const uint4*>(xa + 8 * xstride + (s0 + u) * 64);
-            mma_bf16_16816(c, lo.x, hi.x, lo.y, hi.y, bw[u].x, bw[u].y);
-            mma_bf16_16816(c, lo.z, hi.z, lo.w, hi.w, bw[u].z, bw[u].w);
-          }
-        }
-      }
-      float* dst = kv_a + mat * r + j0 + 2 * qcol;
-      dst[qrow * 2 * r] = c[0];
-      dst[qrow * 2 * r + 1] = c[1];
-      dst[(qrow + 8) * 2 * r] = c[2];
-      dst[(qrow + 8) * 2 * r + 1] = c[3];
-    }
-  }
-  __syncthreads();
-
-  // ---- p = Q_a k_a ------------------------------------------------------------------------------------------------
-  for (int idx = tid; idx < ES_SEQ * G; idx += ES_THREADS) {
-    const int row = idx / G, gi = idx - row * G;
-    float sacc = 0.f;
-    for (int j = 0; j < r; ++j) sacc = fmaf(qa[gi * (r + 1) + j], kv_a[row * 2 * r + j], sacc);
-    pg[idx] = sacc;
-  }
-  __syncthreads();
-
-  // ---- S <- Normalize(S + p v_a^T): a warp per sequence, a state row per 32 lanes ------------------------------------
-  const int jper = (r + 31) >> 5;                    // <= 4 elements of a row per lane
-  for (int row = warp; row < ES_SEQ; row += ES_WARPS) {
-    if (!has[row]) continue;
-    float* S = p.S + ((size_t)l * B + b0 + row) * gr;
-    const float* va = kv_a + row * 2 * r + r;
-    float total = 0.f;
-    for (int g0 = 0; g0 < G; g0 += 8) {
-      float val[8][4];
-#pragma unroll
-      for (int u = 0; u < 8; ++u)
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int gi = g0 + u, j = lane + 32 * jj;
-          val[u][jj] = (gi < G && jj < jper && j < r) ? S[gi * r + j] : 0.f;
-        }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int gi = g0 + u;
-        if (gi >= G) break;
-        const float pw = pg[row * G + gi];
-        float ss = 0.f;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int j = lane + 32 * jj;
-          if (jj < jper && j < r) {
-            val[u][jj] = fmaf(pw, va[j], val[u][jj]);
-            ss = fmaf(val[u][jj], val[u][jj], ss);
-          }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        total += ss;
-        const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int j = lane + 32 * jj;
-          if (jj < jper && j < r) S[gi * r + j] = val[u][jj] * sc;
-        }
-      }
-    }
-    if (p.norm_mode == PTENC_NORM_FROBENIUS) {
-      // the un-normalised sum was stored above; every lane rescales the elements it wrote itself
-      const float sc = 1.f / fmaxf(sqrtf(total), 1e-12f);
-      for (int gi = 0; gi < G; ++gi)
-        for (int j = lane; j < r; j += 32) S[gi * r + j] *= sc;
-    }
-  }
-}
-
 // S[l][b] = S0[l] for every b; zero_s0 != 0 first clears S0[l].
 __global__ void k_broadcast_state(PtencDev p, int layer, int zero_s0) {
   const int gr = p.G * p.r;
@@ -378,36 +205,13 @@ cudaError_t launch_encode_t(ptenc_cache* c, int l0, int nl, const void* Ke, cons
   return cudaGetLastError();
 }
 
-// The one-row-per-sequence tensor-core kernel covers bf16 storage with r a multiple of 8 and d_kv a multiple of 32.
-bool encode_step_usable(const ptenc_cache* c, const void* Ke, int m_max) {
-  const PtencDev& p = c->dev;
-  if (c->cfg.dtype != PTENC_DTYPE_BF16 || (p.r & 7) != 0 || (p.d_kv & 31) != 0) return false;
-  if (Ke == nullptr ? p.E != 1 : m_max != 1) return false;
-  return encode_step_smem(p.G, p.r, p.d_kv) <= 160 * 1024;
-}
-
-cudaError_t launch_encode_step(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve, const int32_t* n_ev,
-                               int m_max, cudaStream_t st) {
-  const PtencDev& p = c->dev;
-  const size_t smem = encode_step_smem(p.G, p.r, p.d_kv);
-  static bool attr_done = false;
-  if (!attr_done && smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k_encode_step_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  const int nblk = (p.B + ES_SEQ - 1) / ES_SEQ;
-  k_encode_step_mma<<<nl * nblk, ES_THREADS, smem, st>>>(p, l0, (const __nv_bfloat16*)Ke, (const __nv_bfloat16*)Ve,
-                                                         n_ev, m_max);
-  c->launches++;
-  return cudaGetLastError();
-}
-
 }  // namespace
 
 cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
                                 const int32_t* n_ev, int m_max, cudaStream_t st) {
-  if (encode_step_usable(c, Ke, m_max)) return launch_encode_step(c, l0, nl, Ke, Ve, n_ev, m_max, st);
+  // one evicted token per sequence: blocks of 16 sequences, projections on warp-level mma
+  if (ptenc_step_e1_usable(c, Ke, m_max)) return ptenc_launch_step_e1(c, l0, nl, false, nullptr, nullptr, nullptr,
+                                                                      Ke, Ve, n_ev, m_max, st);
   // chunks of evicted tokens: the projections are dense contractions -> tensor cores
   if (c->tc_encode && (Ke == nullptr ? c->dev.E : m_max) >= 2 &&
       (Ke == nullptr || (long long)nl * c->cfg.batch * m_max >= 128))

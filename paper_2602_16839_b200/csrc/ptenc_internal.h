@@ -71,6 +71,12 @@ cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void
                                       void* out, float* lse, cudaStream_t st);
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
                                    void* out, float* lse, cudaStream_t st);
+// One evicted token per sequence (E = 1 on the staged path, or caller rows with m_max == 1), bf16: encode alone
+// (append == false) or ring append/evict fused with the encode of the evicted row (append == true; Ke, Ve unused).
+bool ptenc_step_e1_usable(const ptenc_cache* c, const void* Ke, int m_max);
+cudaError_t ptenc_launch_step_e1(ptenc_cache* c, int l0, int nl, bool append, const void* k_new, const void* v_new,
+                                 const uint8_t* active, const void* Ke, const void* Ve, const int32_t* n_ev,
+                                 int m_max, cudaStream_t st);
 // Chunk encoder on tcgen05 (bf16, rank 16/32/64, d_kv % 64 == 0): tensor maps at create time, launch per call.
 bool ptenc_encode_tc_prepare(ptenc_cache* c);
 cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,

@@ -89,15 +89,19 @@ def test_windows_and_chunks(dtype, W, E):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-def test_fused_step_equals_three_calls(dtype):
-    kw = dict(n_layers=3, batch=4, n_q_heads=8, n_kv_heads=2, head_dim=128, window=70, evict_chunk=3,
+@pytest.mark.parametrize("E,batch", [(3, 4), (1, 4), (1, 21)])
+def test_fused_step_equals_three_calls(dtype, E, batch):
+    kw = dict(n_layers=3, batch=batch, n_q_heads=8, n_kv_heads=2, head_dim=128, window=70, evict_chunk=E,
               dtype=dtype, seed=5)
     a, b, c = Pair(pt, **kw), Pair(pt, **kw), Pair(pt, **kw)
     for t in range(160):
         a.step(t, fused=True, all_layers=True)
         b.step(t, fused=False, all_layers=True)
         c.step(t, fused=True, all_layers=False)
-        assert torch.equal(a.out, b.out) and torch.equal(a.out, c.out)
+        assert torch.equal(a.out, b.out)
+        # per-layer calls split the tiles between CTAs at other points than the all-layer call does, so the fp32
+        # partial sums are combined in another order: equal to within a few bf16 ulps, not bit for bit
+        assert float((a.out.float() - c.out.float()).abs().max()) <= 4e-3
     for l in range(3):
         assert torch.equal(a.cache.get_state(l), b.cache.get_state(l))
         assert torch.equal(a.cache.get_state(l), c.cache.get_state(l))
