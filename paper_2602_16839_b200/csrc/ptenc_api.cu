@@ -103,6 +103,26 @@ cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uin
   return rc;
 }
 
+
+// Streams and events of the host-buffer step are made on first use (host objects only, no device memory).
+bool ensure_host_pipeline(ptenc_cache* c) {
+  if (c->st_in != nullptr) return true;
+  bool good = cudaStreamCreateWithFlags(&c->st_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->st_out, cudaStreamNonBlocking) == cudaSuccess;
+  auto mk = [&](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+  mk(&c->ev_start); mk(&c->ev_kv); mk(&c->ev_done);
+  for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) { mk(&c->ev_q[i]); mk(&c->ev_o[i]); }
+  return good;
+}
+
+void release_host_pipeline(ptenc_cache* c) {
+  auto rm = [](cudaEvent_t& e) { if (e != nullptr) { cudaEventDestroy(e); e = nullptr; } };
+  rm(c->ev_start); rm(c->ev_kv); rm(c->ev_done);
+  for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) { rm(c->ev_q[i]); rm(c->ev_o[i]); }
+  if (c->st_in != nullptr) { cudaStreamDestroy(c->st_in); c->st_in = nullptr; }
+  if (c->st_out != nullptr) { cudaStreamDestroy(c->st_out); c->st_out = nullptr; }
+}
+
 }  // namespace
 
 extern "C" {
@@ -141,6 +161,9 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   c->tc_stage_box = 0;
   c->attn_grid = 0;
   c->ev_attn_begin = c->ev_attn_end = nullptr;
+  c->st_in = c->st_out = nullptr;
+  c->ev_start = c->ev_kv = c->ev_done = nullptr;
+  for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) c->ev_q[i] = c->ev_o[i] = nullptr;
 
   PtencDev& d = c->dev;
   char* base = static_cast<char*>(ws);
@@ -180,6 +203,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
 
 int ptenc_cache_destroy(ptenc_cache* c) {
   if (c == nullptr) return PTENC_EINVAL;
+  release_host_pipeline(c);
   delete c;
   return PTENC_OK;
 }
@@ -305,20 +329,68 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
   if ((reinterpret_cast<uintptr_t>(dev_staging) & 255) != 0) return PTENC_EALIGN;
   const HostStaging h = host_staging(c, nl);
   if (staging_bytes < h.total) return PTENC_EWORKSPACE;
+  if (!ensure_host_pipeline(c)) return PTENC_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* sb = static_cast<char*>(dev_staging);
-  if (cudaMemcpyAsync(sb + h.q, q_host, h.qbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
-  if (cudaMemcpyAsync(sb + h.k, k_new_host, h.kvbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
-  if (cudaMemcpyAsync(sb + h.v, v_new_host, h.kvbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PTENC_ECUDA;
+  const PtencDev& d = c->dev;
+  auto good = [](cudaError_t e) { return e == cudaSuccess; };
+
+  // Transfers run on two copy streams forked from `stream` and joined back into it, so that for the caller the
+  // whole call is still ordered on `stream`.  Keys/values go first (the append needs them); the queries and the
+  // outputs move in groups of layers, each group's attention starting as soon as its queries have landed and its
+  // outputs leaving while the next group computes.
+  int ng = (nl + 3) / 4;
+  if (ng > ptenc_cache::HOST_GROUPS_MAX) ng = ptenc_cache::HOST_GROUPS_MAX;
+  if (ng < 1) ng = 1;
+  if (!good(cudaEventRecord(c->ev_start, st)) || !good(cudaStreamWaitEvent(c->st_in, c->ev_start, 0)) ||
+      !good(cudaStreamWaitEvent(c->st_out, c->ev_start, 0)))
+    return PTENC_ECUDA;
   const uint8_t* act = nullptr;
   if (active_host != nullptr) {
-    if (cudaMemcpyAsync(sb + h.active, active_host, c->cfg.batch, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    if (!good(cudaMemcpyAsync(sb + h.active, active_host, c->cfg.batch, cudaMemcpyHostToDevice, c->st_in)))
       return PTENC_ECUDA;
     act = reinterpret_cast<const uint8_t*>(sb + h.active);
   }
-  rc = ptenc_decode_step(c, layer, sb + h.q, sb + h.k, sb + h.v, act, sb + h.out, stream);
-  if (rc != PTENC_OK) return rc;
-  if (cudaMemcpyAsync(out_host, sb + h.out, h.qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PTENC_ECUDA;
+  if (!good(cudaMemcpyAsync(sb + h.k, k_new_host, h.kvbytes, cudaMemcpyHostToDevice, c->st_in)) ||
+      !good(cudaMemcpyAsync(sb + h.v, v_new_host, h.kvbytes, cudaMemcpyHostToDevice, c->st_in)) ||
+      !good(cudaEventRecord(c->ev_kv, c->st_in)))
+    return PTENC_ECUDA;
+  const size_t q_layer = (size_t)d.B * d.d_q * d.elt;
+  for (int g = 0; g < ng; ++g) {
+    const int a0 = g * nl / ng, a1 = (g + 1) * nl / ng;
+    if (!good(cudaMemcpyAsync(sb + h.q + a0 * q_layer, static_cast<const char*>(q_host) + a0 * q_layer,
+                              (size_t)(a1 - a0) * q_layer, cudaMemcpyHostToDevice, c->st_in)) ||
+        !good(cudaEventRecord(c->ev_q[g], c->st_in)))
+      return PTENC_ECUDA;
+  }
+  // a1 + a3 on the caller's stream once the keys/values are on the device
+  if (!good(cudaStreamWaitEvent(st, c->ev_kv, 0))) return PTENC_ECUDA;
+  if (c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0)) {
+    if (!ok(ptenc_launch_step_e1(c, l0, nl, true, sb + h.k, sb + h.v, act, nullptr, nullptr, nullptr, 0, st),
+            "decode_step_host/append_evict+encode", st))
+      return PTENC_ECUDA;
+  } else {
+    if (!ok(ptenc_launch_append_evict(c, l0, nl, sb + h.k, sb + h.v, act, nullptr, nullptr, nullptr, st),
+            "decode_step_host/append_evict", st))
+      return PTENC_ECUDA;
+    if (c->cfg.encode_enabled &&
+        !ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step_host/encode", st))
+      return PTENC_ECUDA;
+  }
+  // a2 group by group
+  for (int g = 0; g < ng; ++g) {
+    const int a0 = g * nl / ng, a1 = (g + 1) * nl / ng;
+    if (!good(cudaStreamWaitEvent(st, c->ev_q[g], 0))) return PTENC_ECUDA;
+    if (!ok(launch_attn(c, l0 + a0, a1 - a0, sb + h.q + a0 * q_layer, act, sb + h.out + a0 * q_layer, nullptr, st),
+            "decode_step_host/attn", st))
+      return PTENC_ECUDA;
+    if (!good(cudaEventRecord(c->ev_o[g], st)) || !good(cudaStreamWaitEvent(c->st_out, c->ev_o[g], 0)) ||
+        !good(cudaMemcpyAsync(static_cast<char*>(out_host) + a0 * q_layer, sb + h.out + a0 * q_layer,
+                              (size_t)(a1 - a0) * q_layer, cudaMemcpyDeviceToHost, c->st_out)))
+      return PTENC_ECUDA;
+  }
+  if (!good(cudaEventRecord(c->ev_done, c->st_out)) || !good(cudaStreamWaitEvent(st, c->ev_done, 0)))
+    return PTENC_ECUDA;
   return PTENC_OK;
 }
 

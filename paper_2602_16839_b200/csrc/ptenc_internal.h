@@ -52,6 +52,10 @@ struct ptenc_cache {
   CUtensorMap tmK, tmV;         // 2-D maps over the rings: rows = L*B*Hkv*W, cols = D
   int attn_grid;                // persistent grid of the fast attention kernel
   cudaEvent_t ev_attn_begin, ev_attn_end;   // one-shot timing hook around the next attention launch
+  // ptenc_decode_step_host: copy streams and events (host objects) that overlap the transfers with the kernels
+  static constexpr int HOST_GROUPS_MAX = 8;
+  cudaStream_t st_in, st_out;
+  cudaEvent_t ev_start, ev_kv, ev_done, ev_q[HOST_GROUPS_MAX], ev_o[HOST_GROUPS_MAX];
   bool tc_encode;               // tensor-core chunk encoder usable for this shape
   CUtensorMap tmWk, tmWv;       // 2-D maps over the encoder weights: rows = L*r, cols = d_kv
   CUtensorMap tmStageK, tmStageV;   // 2-D maps over the staged evicted rows: rows = L*B*E, cols = d_kv

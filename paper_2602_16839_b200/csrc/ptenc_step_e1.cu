@@ -9,8 +9,10 @@
 // bf16 mma (fp32 accumulate), so a layer's weights are read once per 16 sequences instead of once per sequence.
 // Each lane fetches 8 consecutive k-values of its A row (shared memory) and of its B row (W^a, from L2) with one
 // 16-byte load and feeds them to two mma steps; the contraction index is permuted the same way on both operands,
-// which leaves the sum unchanged.  The state rows of a sequence are fetched into registers before the projections
-// start, so their DRAM latency hides behind the weight loads.  Everything after the projections is fp32.
+// which leaves the sum unchanged.  The kernel is a chain of dependent memory round trips, so everything it will
+// need later (its slice of the weights, Q_a, the sequences' state rows) is pulled into L2 with prefetches at the very
+// start, while the ring state and the evicted rows are still on their way; two CTAs fit on an SM so that the whole
+// grid of a 28-layer x 128-sequence step is resident at once.  Everything after the projections is fp32.
 //
 // The same kernel serves ptenc_encode alone (APPEND = false: rows come from the staging area or from the caller).
 #include "ptenc_internal.h"
@@ -20,6 +22,10 @@ namespace {
 constexpr int E1_SEQ = 16;                 // sequences per CTA = rows of the mma tile
 constexpr int E1_THREADS = 512;
 constexpr int E1_WARPS = E1_THREADS / 32;  // one warp per sequence in the row-wise phases
+
+__device__ __forceinline__ void e1_prefetch_l2(const void* ptr) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 
 __device__ __forceinline__ void e1_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                        uint32_t b0, uint32_t b1) {
@@ -55,7 +61,7 @@ __host__ __device__ inline size_t e1_smem_bytes(int G, int r, int d_kv) {
 
 // RJ = ceil(r / 32): state elements of one row held by a lane.
 template <bool APPEND, int RJ>
-__global__ void __launch_bounds__(E1_THREADS, 1)
+__global__ void __launch_bounds__(E1_THREADS, 2)
 k_step_e1(PtencDev p, E1Args a) {
   extern __shared__ __align__(16) uint8_t e1_smem[];
   const int G = p.G, r = p.r, d_kv = p.d_kv, B = p.B, W = p.W;
@@ -78,6 +84,28 @@ k_step_e1(PtencDev p, E1Args a) {
   const size_t ob = (size_t)li * B + b;
   const bool enc_on = p.encode_enabled && p.enc_set[l];
   const int vpr = d_kv >> 3;                         // 16-byte vectors per token row (all KV heads)
+  const int gr = G * r;
+  float* S = p.S + lb * gr;
+  const int tiles_per_map = r >> 3;
+  const int n_tiles = 2 * tiles_per_map;
+  const int n_pairs = d_kv >> 5;                     // 32 k-values per pair of mma steps
+
+  // ---- pull what the later phases read into L2 now (128-byte lines; harmless when it turns out unused) -------------
+  if (enc_on) {
+    if (b < B)
+      for (int i = lane; i * 32 < gr; i += 32) e1_prefetch_l2(S + i * 32);
+    for (int i = tid; i * 32 < gr; i += E1_THREADS) e1_prefetch_l2(p.Qa + (size_t)l * gr + i * 32);
+    for (int item = warp; item < n_tiles * KS; item += E1_WARPS) {
+      const int tile = item % n_tiles, ks = item / n_tiles;
+      const int mat = tile >= tiles_per_map ? 1 : 0;
+      const int j0 = (tile - mat * tiles_per_map) * 8;
+      const int s_lo = ks * n_pairs / KS, s_hi = (ks + 1) * n_pairs / KS;
+      const __nv_bfloat16* w0 = reinterpret_cast<const __nv_bfloat16*>(mat ? p.Wv : p.Wk) + (size_t)l * r * d_kv;
+      const int lines = (s_hi - s_lo + 1) / 2;       // 64 bytes per pair
+      for (int i = lane; i < 8 * lines; i += 32)
+        e1_prefetch_l2(w0 + (size_t)(j0 + (i & 7)) * d_kv + (size_t)s_lo * 32 + (size_t)(i >> 3) * 64);
+    }
+  }
 
   // ---- phase A: the sequence's evicted row -> shared memory (+ staging), the arriving row -> ring ---------------
   int m = 0;
@@ -157,20 +185,7 @@ k_step_e1(PtencDev p, E1Args a) {
   const bool mine = enc_on && m > 0;
   if (lane == 0) has[warp] = mine ? 1 : 0;
 
-  // ---- the first batch of this sequence's state rows, in flight during the projections ----------------------------
   constexpr int NB = 32 / RJ;                        // state rows per batch: 32 registers per lane
-  const int gr = G * r;
-  float* S = p.S + lb * gr;
-  float st[NB][RJ];
-  if (mine) {
-#pragma unroll
-    for (int u = 0; u < NB; ++u)
-#pragma unroll
-      for (int jj = 0; jj < RJ; ++jj) {
-        const int j = lane + 32 * jj;
-        st[u][jj] = (u < G && j < r) ? S[u * r + j] : 0.f;
-      }
-  }
   if (__syncthreads_or(mine ? 1 : 0) == 0) return;   // also orders phase A's shared-memory writes
 
   for (int i = tid; i < gr; i += E1_THREADS) {
@@ -182,9 +197,6 @@ k_step_e1(PtencDev p, E1Args a) {
   {
     const __nv_bfloat16* Wk = reinterpret_cast<const __nv_bfloat16*>(p.Wk) + (size_t)l * r * d_kv;
     const __nv_bfloat16* Wv = reinterpret_cast<const __nv_bfloat16*>(p.Wv) + (size_t)l * r * d_kv;
-    const int tiles_per_map = r >> 3;
-    const int n_tiles = 2 * tiles_per_map;
-    const int n_pairs = d_kv >> 5;                   // 32 k-values per pair of mma steps
     const int qrow = lane >> 2, qcol = lane & 3;
     for (int item = warp; item < n_tiles * KS; item += E1_WARPS) {
       const int tile = item % n_tiles, ks = item / n_tiles;
@@ -240,15 +252,14 @@ k_step_e1(PtencDev p, E1Args a) {
   const float* va = kv_a + warp * 2 * r + r;
   float total = 0.f;
   for (int g0 = 0; g0 < G; g0 += NB) {
-    if (g0 > 0) {
+    float st[NB][RJ];
 #pragma unroll
-      for (int u = 0; u < NB; ++u)
+    for (int u = 0; u < NB; ++u)
 #pragma unroll
-        for (int jj = 0; jj < RJ; ++jj) {
-          const int gi = g0 + u, j = lane + 32 * jj;
-          st[u][jj] = (gi < G && j < r) ? S[gi * r + j] : 0.f;
-        }
-    }
+      for (int jj = 0; jj < RJ; ++jj) {
+        const int gi = g0 + u, j = lane + 32 * jj;
+        st[u][jj] = (gi < G && j < r) ? S[gi * r + j] : 0.f;
+      }
 #pragma unroll
     for (int u = 0; u < NB; ++u) {
       const int gi = g0 + u;
@@ -266,7 +277,7 @@ k_step_e1(PtencDev p, E1Args a) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         total += ss;
-        const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
+        const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? rsqrtf(fmaxf(ss, 1e-24f)) : 1.f;   // 1 / max(|row|, 1e-12)
 #pragma unroll
         for (int jj = 0; jj < RJ; ++jj) {
           const int j = lane + 32 * jj;

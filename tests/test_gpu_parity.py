@@ -295,3 +295,37 @@ def test_tensor_core_encoder_with_caller_rows_and_modes():
             p.check_state(rel=(mode == 2), tol=2e-4 if mode == 2 else TOL_STATE)
         assert p.cache.status() == 0
         p.close()
+
+
+@pytest.mark.parametrize("dtype,L", [("bf16", 9), ("fp32", 2)])
+def test_host_buffer_step_equals_device_step(dtype, L):
+    """ptenc_decode_step_host (pinned host tensors in and out, copies overlapped on internal streams) gives the same
+    outputs, ring and state as ptenc_decode_step on device tensors; also with a mask and for a single layer."""
+    kw = dict(n_layers=L, batch=5, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 64, window=23,
+              evict_chunk=1, dtype=dtype, seed=31)
+    a, b = Pair(pt, **kw), Pair(pt, **kw)
+    staging = torch.empty(b.cache.host_staging_bytes(-1), dtype=torch.uint8, device="cuda")
+    hout = torch.zeros(a.out.shape, dtype=a.out.dtype).pin_memory()
+    rng = np.random.default_rng(3)
+    for t in range(60):
+        active = (rng.random(5) < 0.85).astype(np.uint8) if t % 3 else None
+        a.step(t, active=active)
+        q = b.gen.step_q(t)
+        k, v = b.gen.step_kv(t)
+        qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
+        ah = None if active is None else torch.as_tensor(active).pin_memory()
+        if t % 7 == 5:                                   # layer by layer through the same entry point
+            for l in range(L):
+                b.cache.decode_step_host(l, qh[l], kh[l], vh[l], hout[l], staging, ah)
+        else:
+            b.cache.decode_step_host(-1, qh, kh, vh, hout, staging, ah)
+        torch.cuda.synchronize()
+        m = np.ones(5, bool) if active is None else active.astype(bool)
+        got, want = hout[:, m].float(), a.out[:, m].cpu().float()
+        assert float((got - want).abs().max()) <= (4e-3 if dtype == "bf16" else 1e-6)
+    for l in range(L):
+        assert torch.equal(a.cache.get_state(l), b.cache.get_state(l))
+        for x, y in zip(a.cache.get_ring(l), b.cache.get_ring(l)):
+            assert torch.equal(x, y)
+    assert a.cache.status() == 0 and b.cache.status() == 0
+    a.close(); b.close()
