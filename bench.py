@@ -55,15 +55,36 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def bytes_model(c: dict, evicting: bool = True) -> dict:
-    """Algorithmic bytes of one full-window step (all layers, all sequences active)."""
+def live_after(t: int, W: int, E: int) -> int:
+    """Live tokens of a sequence after its t-th token (0-based) arrived: the ring fills, then every E-th arrival
+    finds it full and evicts E tokens."""
+    return t + 1 if t < W else W - E + 1 + (t - W) % E
+
+
+def evicts_at(t: int, W: int, E: int) -> bool:
+    return t >= W and (t - W) % E == 0
+
+
+def bytes_model(c: dict, E: int = 1, steps=None) -> dict:
+    """Algorithmic bytes (all layers, all sequences active) summed over the given steps (token indices); one
+    full-window evicting step when `steps` is None.  Per layer and sequence: the live K and V rows + q + o for the
+    attention, the arriving K/V rows for the append, and on an evicting step the E evicted K/V rows + the state read
+    and written."""
     L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
     elt = 2 if c["dtype"] == "bf16" else 4
     d_q, d_kv = Hq * D, Hkv * D
-    attn = L * B * (2 * W * d_kv * elt + 2 * d_q * elt)                 # K,V window + q + o
-    append = L * B * 2 * d_kv * elt
-    enc = L * B * (2 * 1 * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) if evicting else 0
-    return {"attn": attn, "step": attn + append + enc}
+    if steps is None:
+        steps = [W]
+        live = [W]
+        ev = [True]
+    else:
+        live = [live_after(t, W, E) for t in steps]
+        ev = [evicts_at(t, W, E) for t in steps]
+    attn = sum(L * B * (2 * n * d_kv * elt + 2 * d_q * elt) for n in live)          # K,V window + q + o
+    append = len(live) * L * B * 2 * d_kv * elt
+    enc = sum(L * B * (2 * E * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) for e in ev if e)
+    return {"attn": attn, "step": attn + append + enc, "attn_per_step": [L * B * (2 * n * d_kv * elt + 2 * d_q * elt)
+                                                                          for n in live]}
 
 
 # ======================================================================================== clocks sampling
@@ -124,14 +145,14 @@ class ClockSampler:
 
 
 # ======================================================================================== CPU oracle legs
-def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1):
+def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1):
     """Times the CPU oracle, as it stands, on 1 layer x n_seq sequences at the full window.
     Returns (seconds per sampled step, threads used)."""
     from oracle.ptenc_oracle import OracleCache
     cc = {**c, "n_layers": 1, "batch": n_seq}
     gen = make_inputs(cc, seed=0, device="cpu")
     orc = OracleCache(n_layers=1, batch=n_seq, n_q_heads=c["n_q_heads"], n_kv_heads=c["n_kv_heads"],
-                      head_dim=c["head_dim"], window=c["window"], evict_chunk=1, n_global=c["n_global"],
+                      head_dim=c["head_dim"], window=c["window"], evict_chunk=E, n_global=c["n_global"],
                       rank=c["rank"])
     P = gen.encoder_params(0)
     orc.set_encoder(0, **{k: v.double().numpy() for k, v in P.items()})
@@ -157,7 +178,7 @@ def run_reference(args, c: dict):
     if rank_env()[0] != 0:
         return
     n_seq = 8 if c["batch"] >= 8 else c["batch"]
-    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup))
+    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup), E=args.evict_chunk)
     value = n_seq / (sec * c["n_layers"])
     sample = (f"1 of {c['n_layers']} layers x {n_seq} of {c['batch']} sequences per step at window {c['window']} "
               f"(full, evicting); tokens/s = {n_seq} / (step time x {c['n_layers']} layers)")
@@ -176,8 +197,10 @@ def run_reference(args, c: dict):
 def config_block(args, c: dict) -> dict:
     return {"workload": args.workload, "n_layers": c["n_layers"], "batch_per_gpu": c["batch"],
             "n_q_heads": c["n_q_heads"], "n_kv_heads": c["n_kv_heads"], "head_dim": c["head_dim"],
-            "window": c["window"], "evict_chunk": 1, "n_global": c["n_global"], "rank": c["rank"],
-            "phase": "steady state: rings full, one eviction + encode per sequence per step",
+            "window": c["window"], "evict_chunk": args.evict_chunk, "n_global": c["n_global"], "rank": c["rank"],
+            "phase": ("steady state: rings full, one eviction + encode per sequence per step" if args.evict_chunk == 1
+                      else f"steady state: rings between {c['window'] - args.evict_chunk + 1} and {c['window']} tokens, "
+                           f"every {args.evict_chunk}-th step evicts and encodes {args.evict_chunk} tokens per sequence"),
             "launch_mode": "all layers per call (layer = -1)",
             "l2": "K/V rings read per step exceed the 126 MB L2 by >100x; no flush needed",
             "parallelism": f"dp{args.gpus} (batch shards, no collective on the path)"}
@@ -223,7 +246,8 @@ def run_gpu(args, c: dict):
 
     L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
     gen = make_inputs(c, seed=shard_seed(rank), device=dev)
-    cfg = pt.make_config(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=1,
+    E = args.evict_chunk
+    cfg = pt.make_config(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=E,
                          n_global=c["n_global"], rank=c["rank"], dtype=c["dtype"], device=local)
     cache = pt.Cache(cfg)
     for l in range(L):
@@ -301,16 +325,20 @@ def run_gpu(args, c: dict):
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
 
     if rank == 0:
-        bm = bytes_model(c)
+        timed_tokens = list(range(W + Wm, W + Wm + K))          # token index arriving at each timed step
+        bm = bytes_model(c, E, timed_tokens)
         peak, peak_kind = measured_peak()
         ms_step = ms_total / K
         attn_avg_ms = sum(attn_ms) / len(attn_ms)
-        attn_gbs = bm["attn"] / (attn_avg_ms * 1e-3) / 1e9
-        step_gbs = bm["step"] / (ms_step * 1e-3) / 1e9
+        attn_gbs = bm["attn"] / (sum(attn_ms) * 1e-3) / 1e9
+        step_gbs = bm["step"] / (ms_total * 1e-3) / 1e9
+        bm["attn"] /= K                                          # per launch / per step averages from here on
+        bm["step"] /= K
         # DRAM bytes per algorithmic byte of the attention kernel, from the ncu capture summarised in
         # profiles/attn_bf16_ncu_full_stress-w2048-b16.md (a smaller batch of the same shape; traffic grows in
         # proportion to the tiles processed), scaled to this launch.
         traffic = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE * bm["attn"] if c["dtype"] == "bf16" else None
+        bm.pop("attn_per_step")
         line = {
             "metric": METRIC, "value": job_tokens_per_s(world, B, K, ms_total), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -332,7 +360,7 @@ def run_gpu(args, c: dict):
         }
         if world == 1 and not args.no_cpu_baseline:
             n_seq, n_steps = min(8, B), args.cpu_steps
-            sec, cores = oracle_sample(c, n_seq, n_steps)
+            sec, cores = oracle_sample(c, n_seq, n_steps, E=E)
             line["cpu_baseline"] = {
                 "value": n_seq / (sec * L), "unit": UNIT, "cores": cores, "kind": "oracle",
                 "sample": (f"oracle decode_step on 1 of {L} layers x {n_seq} of {B} sequences x {n_steps} steps at "
@@ -351,6 +379,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen7b",
                     help="tiny | qwen3b | qwen7b | llama8b | stress-w<W>-b<B>")
+    ap.add_argument("--evict-chunk", type=int, default=1,
+                    help="tokens evicted at once when a ring is full (1 = ring per step, the timed configuration; "
+                         "window/4 is the setting of the paper's runs, Sec. 4.1)")
     ap.add_argument("--cpu-steps", type=int, default=128, help="steps of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -32,7 +32,11 @@ in the tests where the mathematics allows):
   -- parity unpinned.
 * no softmax and no scaling inside the encoder (Eq. (3) has neither);
 * order inside a step: evict, append, attend; the live set never exceeds W;
-* eviction is FIFO by arrival and freed slots are reused FIFO.
+* eviction is FIFO by arrival and freed slots are reused FIFO;
+* pinned question tokens (Sec. 3.3, the sliding-window policy keeps the question; Sec. 4.1): a
+  prompt of n tokens given to `prefill` occupies the first n of the W cache entries for the whole
+  rollout, is attended by every later query, is never evicted and never encoded; the sliding
+  window runs over the remaining W - n entries, and a chunk never exceeds that capacity.
 
 All arithmetic is float64.  Library primitives used as steps: numpy matmul, exp.
 """
@@ -138,7 +142,8 @@ class _Seq:
     """One (layer, sequence) cache: live tokens in arrival order + FIFO free slots."""
 
     def __init__(self, W, Hkv, D):
-        self.live = deque()                 # token indices, oldest first
+        self.pinned = []                    # token indices of the pinned prompt (never evicted)
+        self.live = deque()                 # token indices of the sliding part, oldest first
         self.slot_of = {}                   # token index -> slot
         self.free = deque(range(W))         # free slots, reused in FIFO order
         self.K = np.zeros((W, Hkv, D), F64)
@@ -169,6 +174,26 @@ class OracleCache:
         self.enc[layer] = (Qa, np.asarray(Wk_a, F64), np.asarray(Wv_a, F64))
         self.S[layer] = np.repeat(S0[None], self.B, axis=0)
 
+    # -- prompt: pinned entries -----------------------------------------------------------
+    def prefill(self, layer, K_p, V_p, n_prompt):
+        """The prompt of each sequence enters an empty cache and is pinned: K_p, V_p
+        [B, P_max, Hkv, D], n_prompt [B] tokens each (0 = none), at most W - 1."""
+        K_p = np.asarray(K_p, F64)
+        V_p = np.asarray(V_p, F64)
+        for b in range(self.B):
+            c = self.seqs[layer][b]
+            n = int(n_prompt[b])
+            if n == 0:
+                continue
+            assert c.n_appended == 0 and not c.live and not c.pinned and 0 < n < self.W
+            for i in range(n):
+                s_new = c.free.popleft()
+                c.K[s_new] = K_p[b, i]
+                c.V[s_new] = V_p[b, i]
+                c.pinned.append(i)
+                c.slot_of[i] = s_new
+            c.n_appended = n
+
     # -- a1: append / evict ---------------------------------------------------------------
     def append_evict(self, layer, k_new, v_new, active=None):
         """Token arrives for every active sequence.  Returns per-sequence records:
@@ -185,8 +210,9 @@ class OracleCache:
                 ev_slots.append([])
                 continue
             toks, sl = [], []
-            if len(c.live) == self.W:
-                for _ in range(self.E):
+            capacity = self.W - len(c.pinned)       # entries the sliding part may hold
+            if len(c.live) == capacity:
+                for _ in range(min(self.E, capacity)):
                     t_old = c.live.popleft()
                     s_old = c.slot_of.pop(t_old)
                     toks.append(t_old)
@@ -237,9 +263,9 @@ class OracleCache:
             if active is not None and not active[b]:
                 continue
             c = self.seqs[layer][b]
-            if not c.live:
+            if not c.live and not c.pinned:
                 continue
-            sl = [c.slot_of[t] for t in c.live]
+            sl = [c.slot_of[t] for t in c.pinned] + [c.slot_of[t] for t in c.live]
             o[b], lse[b] = attention_gqa(q[b], c.K[sl], c.V[sl])
         return o, lse
 
@@ -251,8 +277,11 @@ class OracleCache:
         return o, lse, rec
 
     # -- views ---------------------------------------------------------------------------------
+    def pinned_count(self, layer):
+        return np.array([len(self.seqs[layer][b].pinned) for b in range(self.B)], np.int64)
+
     def ring(self, layer):
-        """(oldest-token slot or 0, live count, tokens appended) per sequence."""
+        """(oldest sliding token's slot or 0, sliding tokens held, tokens appended incl. the prompt) per sequence."""
         head = np.zeros((self.B,), np.int64)
         count = np.zeros((self.B,), np.int64)
         n_app = np.zeros((self.B,), np.int64)

@@ -412,12 +412,80 @@ def pin_staged_rows_are_evicted_tokens(mod):
         else:
             assert st is None
 
+# ---------------------------------------------------------------- pinned prompt (Sec. 3.3 policy, Sec. 4.1)
+def pin_prompt_is_pinned_and_window_slides_over_the_rest(mod):
+    """A prompt of n tokens keeps its n cache entries for the whole rollout, every query attends to it, only
+    reasoning tokens are evicted (oldest first, at most the sliding capacity per chunk) and the cache never holds
+    more than W tokens.  Slots and evictions against closed forms, attention against the library routine on the
+    token set worked out from the history."""
+    rng = np.random.default_rng(11)
+    Hq, Hkv, D = 4, 2, 8
+    for W, n, E in [(8, 3, 1), (8, 3, 2), (8, 6, 4), (8, 7, 1), (9, 1, 8), (6, 0, 2), (12, 5, 3)]:
+        cap = W - n
+        Ee = min(E, cap)
+        T = 3 * W + 5
+        c = _mk(mod, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=E, batch=2)
+        Kp = rng.standard_normal((2, max(n, 1), Hkv, D))
+        Vp = rng.standard_normal((2, max(n, 1), Hkv, D))
+        c.prefill(0, Kp, Vp, [n, n])
+        assert list(c.pinned_count(0)) == [n, n]
+        hist_k = [Kp[0, i] for i in range(n)]
+        hist_v = [Vp[0, i] for i in range(n)]
+        for j in range(T):                                  # j-th reasoning token, global index n + j
+            q = rng.standard_normal((2, Hq, D))
+            k = rng.standard_normal((2, Hkv, D))
+            v = rng.standard_normal((2, Hkv, D))
+            o, _, (slots, ev_t, ev_s) = c.decode_step(0, q, k, v)
+            hist_k.append(k[0]); hist_v.append(v[0])
+            assert list(slots) == [n + j % cap] * 2, (W, n, E, j)
+            if j >= cap and (j - cap) % Ee == 0:
+                first = (j - cap) // Ee * Ee
+                want_t = [n + first + i for i in range(Ee)]
+                want_s = [n + (first + i) % cap for i in range(Ee)]
+            else:
+                want_t, want_s = [], []
+            assert ev_t[0] == want_t and ev_s[0] == want_s, (W, n, E, j)
+            assert all(t >= n for t in ev_t[0])             # a prompt token never leaves
+            held = j + 1 if j < cap else cap - Ee + 1 + (j - cap) % Ee
+            head, count, n_app = c.ring(0)
+            assert list(count) == [held] * 2 and list(n_app) == [n + j + 1] * 2 and n + held <= W
+            live = list(range(n)) + list(range(n + j + 1 - held, n + j + 1))
+            ref = _sdpa_last_row(q[0], np.stack([hist_k[t] for t in live]), np.stack([hist_v[t] for t in live]),
+                                 Hq // Hkv)
+            np.testing.assert_allclose(o[0], ref, rtol=0, atol=1e-12)
+
+
+def pin_prompt_rows_never_reach_the_encoder(mod):
+    """Only evicted reasoning tokens are staged for the encoder; with no prompt the cache behaves as before."""
+    rng = np.random.default_rng(12)
+    Hkv, D, W, n = 2, 3, 6, 4
+    c = _mk(mod, n_q_heads=2, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=1)
+    Kp = rng.standard_normal((1, n, Hkv, D))
+    c.prefill(0, Kp, -Kp, [n])
+    ks = rng.standard_normal((9, 1, Hkv, D))
+    for j in range(9):
+        _, ev_t, _ = c.append_evict(0, ks[j], 2 * ks[j])
+        st = c.staged[0][0]
+        if j >= W - n:
+            assert ev_t[0] == [n + j - (W - n)]
+            assert np.array_equal(st[0], ks[j - (W - n), 0].reshape(1, -1))
+            assert np.array_equal(st[1], 2 * ks[j - (W - n), 0].reshape(1, -1))
+        else:
+            assert st is None and ev_t[0] == []
+    a, b = _mk(mod, window=5), _mk(mod, window=5)
+    b.prefill(0, np.zeros((1, 1, 1, 4)), np.zeros((1, 1, 1, 4)), [0])
+    for t in range(12):
+        x = rng.standard_normal((1, 1, 4))
+        ra, rb = a.append_evict(0, x, x), b.append_evict(0, x, x)
+        assert list(ra[0]) == list(rb[0]) and ra[1] == rb[1] and ra[2] == rb[2]
+
 
 PINS = [pin_ring_closed_form, pin_ring_vs_list_model, pin_attention_full_window_is_causal,
         pin_attention_sliding_window, pin_attention_chunked_window, pin_attention_window_one,
         pin_attention_special_cases, pin_attention_gqa_mapping, pin_encode_worked_example,
         pin_encode_exact_rational, pin_encode_identities, pin_encode_recurrence,
-        pin_staged_rows_are_evicted_tokens]
+        pin_staged_rows_are_evicted_tokens, pin_prompt_is_pinned_and_window_slides_over_the_rest,
+        pin_prompt_rows_never_reach_the_encoder]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -451,11 +519,15 @@ MUTATIONS = {
     "encoder_softmax_scale": ("P = np.asarray(Qa, F64) @ Ka.T ", "P = np.asarray(Qa, F64) @ Ka.T / np.sqrt(Ka.shape[1]) "),
     "drop_accumulate": ("normalize(np.asarray(S, F64) + context_state(", "normalize(context_state("),
     "normalize_axis": ("n = np.sqrt(np.sum(S * S, axis=-1, keepdims=True))", "n = np.sqrt(np.sum(S * S, axis=0, keepdims=True))"),
-    "evict_after_append": ("if len(c.live) == self.W:", "if len(c.live) > self.W:"),
-    "evict_one_too_early": ("if len(c.live) == self.W:", "if len(c.live) == self.W - 1 and self.W > 1:"),
+    "evict_after_append": ("if len(c.live) == capacity:", "if len(c.live) > capacity:"),
+    "evict_one_too_early": ("if len(c.live) == capacity:", "if len(c.live) == capacity - 1 and capacity > 1:"),
     "lifo_free_slots": ("s_new = c.free.popleft()", "s_new = c.free.pop()"),
     "evict_newest": ("t_old = c.live.popleft()", "t_old = c.live.pop()"),
-    "new_token_not_attended": ("sl = [c.slot_of[t] for t in c.live]", "sl = [c.slot_of[t] for t in list(c.live)[:-1]] or [c.slot_of[c.live[-1]]]"),
+    "new_token_not_attended": ("+ [c.slot_of[t] for t in c.live]", "+ ([c.slot_of[t] for t in list(c.live)[:-1]] or [c.slot_of[c.live[-1]]])"),
+    "prompt_not_attended": ("sl = [c.slot_of[t] for t in c.pinned] + ", "sl = "),
+    "prompt_gets_evicted": ("capacity = self.W - len(c.pinned)", "capacity = self.W - len(c.pinned); c.live.extendleft(reversed(c.pinned)); c.pinned = []"),
+    "window_ignores_prompt": ("capacity = self.W - len(c.pinned) ", "capacity = self.W "),
+    "chunk_exceeds_capacity": ("for _ in range(min(self.E, capacity)):", "for _ in range(self.E):"),
     "stale_v": ("c.V[s_new] = v_new[b]", "c.V[s_new] = k_new[b]"),
     "encode_ignores_disable": ("if not self.encode_enabled:\n            return", "if False:\n            return"),
     "lse_without_max": ("return o, smax + np.log(z)", "return o, np.log(z)"),
