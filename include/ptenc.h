@@ -109,6 +109,21 @@ PTENC_API int ptenc_set_encoder(ptenc_cache* c, int layer, const void* Wq_a, con
                       const void* q_g, const void* k_g /*nullable*/, const void* v_g /*nullable*/,
                       void* stream);
 
+/* Pinned prompt entries (Sec. 3.3: the sliding-window policy keeps the question tokens; Sec. 4.1).  For every
+ * sequence with n_prompt[b] > 0 the first n_prompt[b] rows of K_p, V_p [B, p_max, H_kv, D] (leading [L] when
+ * layer == -1) are stored in slots [0, n_prompt[b]) of the sequence's cache and stay there for the whole rollout:
+ * every later query attends to them, they are never evicted and never reach the encoder; the ring of
+ * ptenc_append_evict then runs over the remaining W - n_prompt[b] slots, and a chunk of evicted tokens never exceeds
+ * that capacity.  n_prompt: device int32 [B], the same for every layer.  The sequence must be empty (fresh or reset)
+ * and 0 < n_prompt[b] <= min(p_max, W - 1); a sequence that breaks this is left untouched and the device status word
+ * gets PTENC_ST_BAD_INDEX (2).  n_prompt[b] == 0 leaves the sequence as it is.  Token indices reported by
+ * ptenc_append_evict count the prompt tokens first. */
+PTENC_API int ptenc_prefill(ptenc_cache* c, int layer, const void* K_p, const void* V_p,
+                            const int32_t* n_prompt /*[B]*/, int32_t p_max, void* stream);
+
+/* Copies one layer's pinned-entry counts to n_pinned [B] (device int32). */
+PTENC_API int ptenc_get_pinned(ptenc_cache* c, int layer, int32_t* n_pinned, void* stream);
+
 /* a1.  For each active sequence the token with key/value k_new/v_new [B, H_kv, D] arrives.  If the
  * sequence already holds W tokens, its E oldest tokens are evicted first (FIFO): their K/V rows are
  * copied, oldest first and KV heads concatenated, to the staging area for ptenc_encode, and their slots
@@ -155,8 +170,9 @@ PTENC_API int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_ho
                                      const void* v_new_host, const uint8_t* active_host, void* out_host,
                                      void* dev_staging, size_t staging_bytes, void* stream);
 
-/* Copies one layer's ring state to device arrays [B] (each nullable): head = slot of the oldest live
- * token, count = live tokens, n_appended = tokens ever appended. */
+/* Copies one layer's ring state to device arrays [B] (each nullable): head = slot of the oldest token of the
+ * sliding part, counted from the first slot after the pinned entries; count = tokens in the sliding part;
+ * n_appended = tokens ever appended (pinned prompt included). */
 PTENC_API int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* count, int64_t* n_appended,
                    void* stream);
 

@@ -21,7 +21,7 @@ DTYPE_FP32, DTYPE_BF16 = 0, 1
 NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
-           "ptenc_set_encoder", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
+           "ptenc_set_encoder", "ptenc_prefill", "ptenc_get_pinned", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
            "ptenc_host_staging_bytes", "ptenc_decode_step_host",
            "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count", "ptenc_strerror"]
 
@@ -41,7 +41,7 @@ class PtencError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2602_16839_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2602_16839_b200/build.py` "
             "(there is no CPU or PyTorch fallback for this path)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
@@ -51,6 +51,8 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_cache_destroy.argtypes = [vp]
     lib.ptenc_cache_reset.argtypes = [vp, vp, vp]
     lib.ptenc_set_encoder.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.ptenc_prefill.argtypes = [vp, i32, vp, vp, vp, ctypes.c_int32, vp]
+    lib.ptenc_get_pinned.argtypes = [vp, i32, vp, vp]
     lib.ptenc_append_evict.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.ptenc_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.ptenc_encode.argtypes = [vp, i32, vp, vp, vp, ctypes.c_int32, vp]
@@ -156,6 +158,15 @@ class Cache:
     def set_encoder(self, layer, Wq_a, Wk_a, Wv_a, q_g, k_g=None, v_g=None):
         _check(lib.ptenc_set_encoder(self._h, layer, _ptr(Wq_a), _ptr(Wk_a), _ptr(Wv_a), _ptr(q_g), _ptr(k_g),
                                      _ptr(v_g), _stream()), "ptenc_set_encoder")
+
+    def prefill(self, layer, K_p, V_p, n_prompt, p_max):
+        _check(lib.ptenc_prefill(self._h, layer, _ptr(K_p), _ptr(V_p), _ptr(n_prompt), int(p_max), _stream()),
+               "ptenc_prefill")
+
+    def get_pinned(self, layer):
+        n = torch.empty(self.cfg.batch, dtype=torch.int32, device=self.device)
+        _check(lib.ptenc_get_pinned(self._h, layer, _ptr(n), _stream()), "ptenc_get_pinned")
+        return n
 
     def append_evict(self, layer, k_new, v_new, active=None, slot_out=None, evict_first_out=None,
                      n_evicted_out=None):

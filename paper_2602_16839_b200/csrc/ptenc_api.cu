@@ -14,7 +14,7 @@ constexpr int PART_SLOTS = 2048;      // split partial slots (two per CTA of the
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t K, V, head, count, n_app, stageK, stageV, n_staged, evict_first, S, S0, Qa, Wk, Wv, enc_set,
+  size_t K, V, head, count, n_app, n_sink, stageK, stageV, n_staged, evict_first, S, S0, Qa, Wk, Wv, enc_set,
       part_acc, part_ml, tickets, status, total;
 };
 
@@ -51,6 +51,7 @@ Layout make_layout(const ptenc_config* c) {
   o.head = take(L * B * 4);
   o.count = take(L * B * 4);
   o.n_app = take(L * B * 8);
+  o.n_sink = take(L * B * 4);
   o.stageK = take(L * B * E * d_kv * elt);
   o.stageV = take(L * B * E * d_kv * elt);
   o.n_staged = take(L * B * 4);
@@ -176,6 +177,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   d.head = reinterpret_cast<int*>(base + lay.head);
   d.count = reinterpret_cast<int*>(base + lay.count);
   d.n_app = reinterpret_cast<long long*>(base + lay.n_app);
+  d.n_sink = reinterpret_cast<int*>(base + lay.n_sink);
   d.stageK = base + lay.stageK; d.stageV = base + lay.stageV;
   d.n_staged = reinterpret_cast<int*>(base + lay.n_staged);
   d.evict_first = reinterpret_cast<long long*>(base + lay.evict_first);
@@ -228,6 +230,24 @@ int ptenc_set_encoder(ptenc_cache* c, int layer, const void* Wq_a, const void* W
   if (cudaMemcpyAsync(d.Wv + (size_t)layer * wbytes, Wv_a, wbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return PTENC_ECUDA;
   return ptenc_launch_set_encoder(c, layer, Wq_a, q_g, k_g, v_g, st) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_prefill(ptenc_cache* c, int layer, const void* K_p, const void* V_p, const int32_t* n_prompt,
+                  int32_t p_max, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (K_p == nullptr || V_p == nullptr || n_prompt == nullptr || p_max < 1) return PTENC_EINVAL;
+  if (misaligned(K_p) || misaligned(V_p)) return PTENC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return ok(ptenc_launch_prefill(c, l0, nl, K_p, V_p, n_prompt, p_max, st), "prefill", st) ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_get_pinned(ptenc_cache* c, int layer, int32_t* n_pinned, void* stream) {
+  if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers || n_pinned == nullptr) return PTENC_EINVAL;
+  const size_t B = c->cfg.batch;
+  return cudaMemcpyAsync(n_pinned, c->dev.n_sink + layer * B, B * 4, cudaMemcpyDeviceToDevice,
+                         static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_append_evict(ptenc_cache* c, int layer, const void* k_new, const void* v_new, const uint8_t* active,

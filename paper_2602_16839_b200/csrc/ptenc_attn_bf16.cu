@@ -116,19 +116,29 @@ __device__ __forceinline__ void consumer_sync(int nthreads) {
 }
 
 // ------------------------------------------------------------------------------------------------ schedule
-// Live tiles of one ring: `nt` tiles starting at tile t0, cyclic over the n_t tiles of the ring.
+// Tiles of one ring that hold live slots.  Live slots are the pinned entries [0, sink) and the `count` slots of the
+// sliding part, which starts at slot sink + head and wraps inside [sink, W).  As a set of slots that is a low
+// interval [0, end1) (pinned entries plus the wrapped tail of the sliding part) and a high interval starting at
+// sink + head.  The unit's tiles are enumerated high interval first: tile t0 + i for i < len2, then tile i - len2.
 template <int TILE_N>
-__device__ __forceinline__ int ring_tiles(int head, int count, int W, int n_t, int* t0) {
-  *t0 = head / TILE_N;
-  if (count <= 0) return 0;
-  const int last = head + count - 1;
-  if (last < W) return last / TILE_N - *t0 + 1;
-  const int n = (n_t - *t0) + (last - W) / TILE_N + 1;
-  return n < n_t ? n : n_t;
+__device__ __forceinline__ int live_tiles(int sink, int head, int count, int W, int* t0, int* len2) {
+  int end1 = sink, n2 = 0;
+  if (count > 0) {
+    const int first = (W - sink) - head;            // sliding slots before the wrap
+    if (count > first) { end1 = sink + (count - first); n2 = first; } else n2 = count;
+  }
+  const int e1 = end1 > 0 ? (end1 - 1) / TILE_N : -1;
+  if (n2 == 0) { *t0 = 0; *len2 = 0; return e1 + 1; }
+  const int s2 = sink + head;
+  const int t2 = s2 / TILE_N, e2 = (s2 + n2 - 1) / TILE_N;
+  *t0 = t2;
+  *len2 = e2 - t2 + 1;
+  const int low = (e1 + 1) < t2 ? (e1 + 1) : t2;    // low-interval tiles not already counted in the high run
+  return *len2 + low;
 }
 
 struct Entry {          // one (layer, sequence) of the call
-  int head, count, nt, t0;
+  int head, count, sink, nt, t0, len2;
 };
 
 template <int D, int TILE_N, int NW, int STAGES>
@@ -193,13 +203,20 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   // ---- schedule: total tile count and this CTA's starting entry ------------------------------------
   auto load_entry = [&](int e) -> Entry {
     Entry en;
-    if (e < 0 || e >= n_ent) { en.head = en.count = en.nt = en.t0 = 0; return en; }
+    en.head = en.count = en.sink = en.nt = en.t0 = en.len2 = 0;
+    if (e < 0 || e >= n_ent) return en;
     const int li = e / B, b = e - li * B;
     const size_t lb = (size_t)(l0 + li) * B + b;
+    if (active != nullptr && active[b] == 0) return en;          // inactive: no tiles
     en.head = p.head[lb];
-    en.count = (active != nullptr && active[b] == 0) ? 0 : p.count[lb];
-    if (en.head < 0 || en.head >= W || en.count < 0 || en.count > W) { en.head = 0; en.count = 0; }
-    en.nt = ring_tiles<TILE_N>(en.head, en.count, W, n_t, &en.t0);
+    en.count = p.count[lb];
+    en.sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;
+    const int cap = W - en.sink;
+    if (en.sink < 0 || cap < 1 || en.head < 0 || en.head >= cap || en.count < 0 || en.count > cap) {
+      en.head = en.count = en.sink = 0;
+      return en;
+    }
+    en.nt = live_tiles<TILE_N>(en.sink, en.head, en.count, W, &en.t0, &en.len2);
     return en;
   };
   const int chunk = (n_ent + NTHREADS - 1) / NTHREADS;
@@ -247,7 +264,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   int h = (int)((t_begin - pe_start * Hkv) / en.nt);
   long long ub = pe_start * Hkv + (long long)h * en.nt;
   Entry nxt;                                             // prefetched entry e + 1
-  nxt.nt = 0; nxt.head = nxt.count = nxt.t0 = 0;
+  nxt.nt = 0; nxt.head = nxt.count = nxt.sink = nxt.t0 = nxt.len2 = 0;
   if (e + 1 < n_ent) nxt = load_entry(e + 1);
 
   auto advance = [&]() {                                 // to the next unit with tiles
@@ -288,8 +305,8 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         }
         const long long row0 = ((long long)lb * Hkv + h) * W;
         for (long long t = lo; t < hi; ++t, ++n) {
-          int j = en.t0 + (int)(t - ub);
-          if (j >= n_t) j -= n_t;
+          const int iu = (int)(t - ub);                  // i-th tile of the unit
+          const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
           const uint32_t s = n % STAGES;
           const long long yy = row0 + (long long)j * TILE_N;
           if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
@@ -334,7 +351,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     const long long hi = (ub + en.nt) < t_end ? (ub + en.nt) : t_end;
     const int n_mine = (int)(hi - lo);
     const int li = e / B, b = e - li * B;
-    const int head = en.head, count = en.count;
+    const int head = en.head, count = en.count, sink = en.sink, cap = W - en.sink;
 
     // ---- Q fragments (A operand, rows = heads; rows >= g are zero) ------------------------------------
     uint32_t qa[KSTEPS][2];
@@ -365,8 +382,8 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     for (int i = i0; i < n_mine; i += NW) {
       const uint32_t seq = n + i;
       const uint32_t s = seq % STAGES;
-      int j = en.t0 + (int)(lo - ub) + i;
-      if (j >= n_t) j -= n_t;
+      const int iu = (int)(lo - ub) + i;
+      const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
       if (misc[0] == 0 && !mbar_wait(bar_full + 8 * s, (seq / STAGES) & 1)) {
         atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
         misc[0] = 1;
@@ -393,19 +410,26 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         }
       }
       // ---- mask slots that hold no live token -------------------------------------------------------------
+      // live: a pinned entry (slot < sink), or a sliding slot whose distance from the head is below count
       const int slot0 = j * TILE_N;
-      int d0 = slot0 - head;
-      if (d0 < 0) d0 += W;
-      const bool full = (slot0 + TILE_N <= W) && (count == W || d0 + TILE_N <= count);
+      bool full = false;
+      if (slot0 + TILE_N <= sink) {
+        full = true;
+      } else if (slot0 >= sink && slot0 + TILE_N <= W) {
+        int d0 = slot0 - sink - head;
+        if (d0 < 0) d0 += cap;
+        full = (count == cap) || (d0 + TILE_N <= count);
+      }
       if (!full) {
 #pragma unroll
         for (int nt = 0; nt < NT8; ++nt) {
 #pragma unroll
           for (int x = 0; x < 2; ++x) {
             const int slot = slot0 + 8 * nt + 2 * qc + x;
-            int dd = slot - head;
-            if (dd < 0) dd += W;
-            if (slot >= W || dd >= count) sc[nt][x] = -INFINITY;
+            int dd = slot - sink - head;
+            if (dd < 0) dd += cap;
+            const bool live = slot < sink || (slot < W && dd < count);
+            if (!live) sc[nt][x] = -INFINITY;
           }
         }
       }

@@ -28,7 +28,9 @@ k_attn_generic(PtencDev p, int l0, const T* __restrict__ q, const uint8_t* __res
   if (active != nullptr && active[b] == 0) return;
   const size_t lb = (size_t)l * p.B + b;
   const int head = p.head[lb], count = p.count[lb];
-  if (count <= 0) return;
+  const int sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;      // pinned prompt entries in slots [0, sink)
+  const int cap = W - sink;
+  if (count + sink <= 0) return;
   const int hkv = hq / p.g;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -45,9 +47,13 @@ k_attn_generic(PtencDev p, int l0, const T* __restrict__ q, const uint8_t* __res
 #pragma unroll
   for (int j = 0; j < AG_MAXJ; ++j) acc[j] = 0.f;
 
-  for (int i = warp; i < count; i += AG_WARPS) {
-    int slot = head + i;
-    if (slot >= W) slot -= W;
+  for (int i = warp; i < sink + count; i += AG_WARPS) {
+    int slot = i;
+    if (i >= sink) {
+      slot = head + (i - sink);
+      if (slot >= cap) slot -= cap;
+      slot += sink;
+    }
     const T* kr = Kb + (size_t)slot * D;
     const T* vr = Vb + (size_t)slot * D;
     float s = 0.f;

@@ -23,7 +23,9 @@ struct PtencDev {
   char* V;
   int* head;                    // [L][B] slot of the oldest live token
   int* count;                   // [L][B] live tokens
-  long long* n_app;             // [L][B] tokens ever appended
+  long long* n_app;             // [L][B] tokens ever appended (pinned prompt included)
+  int* n_sink;                  // [L][B] pinned prompt entries: slots [0, n_sink); the ring runs over the rest.
+                                //        May be null (= no pinned entries anywhere).
   char* stageK;                 // [L][B][E][d_kv] evicted rows of the last append, oldest first
   char* stageV;
   int* n_staged;                // [L][B] rows staged by the last append (0 or E)
@@ -67,6 +69,8 @@ cudaError_t ptenc_launch_append_evict(ptenc_cache* c, int l0, int nl, const void
                                       const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
                                       int32_t* n_evicted_out, cudaStream_t st);
 cudaError_t ptenc_launch_reset(ptenc_cache* c, const uint8_t* seq_mask, cudaStream_t st);
+cudaError_t ptenc_launch_prefill(ptenc_cache* c, int l0, int nl, const void* K_p, const void* V_p,
+                                 const int32_t* n_prompt, int p_max, cudaStream_t st);
 cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
                                 const int32_t* n_ev, int m_max, cudaStream_t st);
 cudaError_t ptenc_launch_set_encoder(ptenc_cache* c, int layer, const void* Wq, const void* qg,

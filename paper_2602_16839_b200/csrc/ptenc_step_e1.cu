@@ -116,19 +116,22 @@ k_step_e1(PtencDev p, E1Args a) {
       if (act) {
         int head = p.head[lb], count = p.count[lb];
         const long long n = p.n_app[lb];
-        if (head < 0 || head >= W || count < 0 || count > W) {
+        const int ns = p.n_sink[lb];                 // pinned prompt entries; the ring runs over slots [ns, W)
+        const int cap = W - ns;
+        if (ns < 0 || cap < 1 || head < 0 || head >= cap || count < 0 || count > cap) {
           atomicOr(p.status, PTENC_ST_BAD_INDEX);
         } else {
           long long first = -1;
-          if (count == W) {                          // full: the oldest token leaves, its slot is reused at once
+          if (count == cap) {                        // full: the oldest token leaves, its slot is reused at once
             m = 1;
-            ev_slot = head;
+            ev_slot = ns + head;
             first = n - count;
-            head = head + 1 == W ? 0 : head + 1;
+            head = head + 1 == cap ? 0 : head + 1;
             count -= 1;
           }
           new_slot = head + count;
-          if (new_slot >= W) new_slot -= W;
+          if (new_slot >= cap) new_slot -= cap;
+          new_slot += ns;
           p.head[lb] = head;
           p.count[lb] = count + 1;
           p.n_app[lb] = n + 1;

@@ -46,15 +46,28 @@ class Pair:
     def close(self):
         self.cache.close()
 
+    def prefill(self, n_prompt, p_max, tensor_id=50):
+        """Pins a synthetic prompt of n_prompt[b] tokens per sequence on both sides."""
+        shape = (self.L, self.B, p_max, self.Hkv, self.D)
+        Kp = self.gen.generic(tensor_id, 0, shape, 1.0)
+        Vp = self.gen.generic(tensor_id + 1, 0, shape, 1.0)
+        n_dev = torch.as_tensor(np.asarray(n_prompt), dtype=torch.int32, device="cuda:0")
+        self.cache.prefill(-1, Kp, Vp, n_dev, p_max)
+        for l in range(self.L):
+            self.orc.prefill(l, np64(Kp[l]), np64(Vp[l]), n_prompt)
+
     def check_ring(self):
         for l in range(self.L):
             head, count, n_app = self.cache.get_ring(l)
+            pinned = self.cache.get_pinned(l).cpu().numpy()
             oh, oc, on = self.orc.ring(l)
             count = count.cpu().numpy()
             assert np.array_equal(count, oc), (l, count, oc)
             assert np.array_equal(n_app.cpu().numpy(), on)
+            assert np.array_equal(pinned, self.orc.pinned_count(l))
             live = oc > 0
-            assert np.array_equal(head.cpu().numpy()[live], oh[live])
+            # the library counts the head from the first slot after the pinned entries
+            assert np.array_equal((head.cpu().numpy() + pinned)[live], oh[live])
 
     def check_state(self, tol=TOL_STATE, rel=False):
         worst = 0.0

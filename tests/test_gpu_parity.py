@@ -329,3 +329,58 @@ def test_host_buffer_step_equals_device_step(dtype, L):
             assert torch.equal(x, y)
     assert a.cache.status() == 0 and b.cache.status() == 0
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("W,E,prompts", [(37, 1, [0, 1, 17, 36, 5]), (96, 24, [0, 33, 64, 95, 80]),
+                                         (200, 50, [130, 7, 0, 199, 64])])
+def test_pinned_prompt_and_sliding_window_over_the_rest(dtype, W, E, prompts):
+    """Prompt lengths from none to W - 1 (a single sliding slot), chunks larger than the remaining capacity, tiles
+    that straddle the end of the pinned part: outputs, eviction reports, ring and state against the oracle."""
+    p = Pair(pt, n_layers=2, batch=5, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 64,
+             window=W, evict_chunk=E, dtype=dtype, seed=W, n_global=16, rank=16)
+    p.prefill(prompts, max(prompts))
+    p.check_ring()
+    B = 5
+    slot = torch.empty(B, dtype=torch.int32, device="cuda")
+    first = torch.empty(B, dtype=torch.int64, device="cuda")
+    nev = torch.empty(B, dtype=torch.int32, device="cuda")
+    out1 = torch.zeros(B, 8, p.D, dtype=p.cache.torch_dtype, device="cuda")
+    for t in range(2 * W + 9):
+        if t % 4 == 3:                                    # three separate calls on layer 1, index reports checked
+            q = p.gen.step_q(t)
+            k, v = p.gen.step_kv(t)
+            p.cache.decode_step(0, q[0], k[0], v[0], p.out[0])
+            p.cache.append_evict(1, k[1], v[1], None, slot, first, nev)
+            p.cache.encode(1)
+            p.cache.decode_attn(1, q[1], out1)
+            for l in range(2):
+                o_ref, _, (slots, ev_t, ev_s) = p.orc.decode_step(l, np64(q[l]), np64(k[l]), np64(v[l]))
+                got = p.out[0] if l == 0 else out1
+                assert np.abs(np64(got) - o_ref).max() <= TOL_OUT[dtype]
+            assert np.array_equal(slot.cpu().numpy(), slots)
+            assert first.cpu().tolist() == [e[0] if e else -1 for e in ev_t]
+            assert nev.cpu().tolist() == [len(e) for e in ev_t]
+        else:
+            p.step(t)
+        if t % 11 == 0:
+            p.check_ring()
+    p.check_ring()
+    p.check_state()
+    assert p.cache.status() == 0
+    p.close()
+
+
+def test_prefill_misuse_sets_the_status_word():
+    p = Pair(pt, n_layers=1, batch=3, n_q_heads=4, n_kv_heads=1, head_dim=64, window=8, dtype="bf16", seed=1)
+    p.step(0)                                              # sequences are no longer empty
+    Kp = torch.zeros(1, 3, 8, 1, 64, dtype=torch.bfloat16, device="cuda")
+    n = torch.tensor([2, 0, 0], dtype=torch.int32, device="cuda")
+    p.cache.prefill(-1, Kp, Kp, n, 8)
+    assert p.cache.status() == 2 and p.cache.get_pinned(0).tolist() == [0, 0, 0]
+    p.cache.reset()                                        # clears rings, pinned counts and the status word
+    assert p.cache.status() == 0
+    n = torch.tensor([8, 3, 0], dtype=torch.int32, device="cuda")      # 8 = W: no slot left for the sliding part
+    p.cache.prefill(-1, Kp, Kp, n, 8)
+    assert p.cache.status() == 2 and p.cache.get_pinned(0).tolist() == [0, 3, 0]
+    p.close()
