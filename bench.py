@@ -55,17 +55,20 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def live_after(t: int, W: int, E: int) -> int:
-    """Live tokens of a sequence after its t-th token (0-based) arrived: the ring fills, then every E-th arrival
-    finds it full and evicts E tokens."""
-    return t + 1 if t < W else W - E + 1 + (t - W) % E
+def live_after(t: int, W: int, E: int, P: int = 0) -> int:
+    """Tokens a sequence holds after its t-th decoded token (0-based) arrived: P pinned prompt tokens plus the sliding
+    part, which fills its W - P slots and then, on every E-th arrival, is found full and evicts E tokens."""
+    cap = W - P
+    E = min(E, cap)
+    return P + (t + 1 if t < cap else cap - E + 1 + (t - cap) % E)
 
 
-def evicts_at(t: int, W: int, E: int) -> bool:
-    return t >= W and (t - W) % E == 0
+def evicts_at(t: int, W: int, E: int, P: int = 0) -> bool:
+    cap = W - P
+    return t >= cap and (t - cap) % min(E, cap) == 0
 
 
-def bytes_model(c: dict, E: int = 1, steps=None) -> dict:
+def bytes_model(c: dict, E: int = 1, steps=None, P: int = 0) -> dict:
     """Algorithmic bytes (all layers, all sequences active) summed over the given steps (token indices); one
     full-window evicting step when `steps` is None.  Per layer and sequence: the live K and V rows + q + o for the
     attention, the arriving K/V rows for the append, and on an evicting step the E evicted K/V rows + the state read
@@ -78,11 +81,11 @@ def bytes_model(c: dict, E: int = 1, steps=None) -> dict:
         live = [W]
         ev = [True]
     else:
-        live = [live_after(t, W, E) for t in steps]
-        ev = [evicts_at(t, W, E) for t in steps]
+        live = [live_after(t, W, E, P) for t in steps]
+        ev = [evicts_at(t, W, E, P) for t in steps]
     attn = sum(L * B * (2 * n * d_kv * elt + 2 * d_q * elt) for n in live)          # K,V window + q + o
     append = len(live) * L * B * 2 * d_kv * elt
-    enc = sum(L * B * (2 * E * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) for e in ev if e)
+    enc = sum(L * B * (2 * min(E, W - P) * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) for e in ev if e)
     return {"attn": attn, "step": attn + append + enc, "attn_per_step": [L * B * (2 * n * d_kv * elt + 2 * d_q * elt)
                                                                           for n in live]}
 
@@ -197,7 +200,7 @@ def run_reference(args, c: dict):
 def config_block(args, c: dict) -> dict:
     return {"workload": args.workload, "n_layers": c["n_layers"], "batch_per_gpu": c["batch"],
             "n_q_heads": c["n_q_heads"], "n_kv_heads": c["n_kv_heads"], "head_dim": c["head_dim"],
-            "window": c["window"], "evict_chunk": args.evict_chunk, "n_global": c["n_global"], "rank": c["rank"],
+            "window": c["window"], "evict_chunk": args.evict_chunk, "pinned_prompt": args.prompt_len, "n_global": c["n_global"], "rank": c["rank"],
             "phase": ("steady state: rings full, one eviction + encode per sequence per step" if args.evict_chunk == 1
                       else f"steady state: rings between {c['window'] - args.evict_chunk + 1} and {c['window']} tokens, "
                            f"every {args.evict_chunk}-th step evicts and encodes {args.evict_chunk} tokens per sequence"),
@@ -262,8 +265,15 @@ def run_gpu(args, c: dict):
         pool.append((gen.step_q(t), k, v))
     out = torch.empty_like(pool[0][0])
 
-    # fill the rings (untimed): W steps reach the full window; warm-up steps then run in steady state
-    for t in range(W):
+    # pinned prompt (Sec. 3.3 / 4.1 policy), then fill the rings (untimed): the sliding part reaches its capacity;
+    # warm-up steps then run in steady state
+    P = args.prompt_len
+    if P > 0:
+        Kp = gen.generic(50, 0, (L, B, P, Hkv, D), 1.0)
+        Vp = gen.generic(51, 0, (L, B, P, Hkv, D), 1.0)
+        cache.prefill(-1, Kp, Vp, torch.full((B,), P, dtype=torch.int32, device=dev), P)
+        del Kp, Vp
+    for t in range(W - P):
         q, k, v = pool[t % R]
         cache.append_evict(-1, k, v)
     torch.cuda.synchronize()
@@ -325,8 +335,8 @@ def run_gpu(args, c: dict):
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
 
     if rank == 0:
-        timed_tokens = list(range(W + Wm, W + Wm + K))          # token index arriving at each timed step
-        bm = bytes_model(c, E, timed_tokens)
+        timed_tokens = list(range(W - P + Wm, W - P + Wm + K))  # decoded-token index arriving at each timed step
+        bm = bytes_model(c, E, timed_tokens, P)
         peak, peak_kind = measured_peak()
         ms_step = ms_total / K
         attn_avg_ms = sum(attn_ms) / len(attn_ms)
@@ -382,6 +392,9 @@ def main():
     ap.add_argument("--evict-chunk", type=int, default=1,
                     help="tokens evicted at once when a ring is full (1 = ring per step, the timed configuration; "
                          "window/4 is the setting of the paper's runs, Sec. 4.1)")
+    ap.add_argument("--prompt-len", type=int, default=0,
+                    help="tokens of a pinned prompt per sequence (kept for the whole rollout; the window slides over "
+                         "the remaining slots)")
     ap.add_argument("--cpu-steps", type=int, default=128, help="steps of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -42,6 +42,14 @@ class _IntOracle:
                              evict_chunk=E, n_global=1, rank=1)
         self.evicted = [[] for _ in self.seqs]           # token indices in eviction order
 
+    def prefill(self, n_prompt_all):
+        n = [int(n_prompt_all[b]) for b in self.seqs]
+        z = np.zeros((len(self.seqs), max(max(n), 1), 1, 1))
+        self.o.prefill(0, z, z, n)
+
+    def pinned(self, i):
+        return list(self.o.seqs[0][i].pinned)
+
     def step(self, active_all):
         act = None if active_all is None else [int(active_all[b]) for b in self.seqs]
         z = np.zeros((len(self.seqs), 1, 1))
@@ -222,6 +230,74 @@ def test_whole_rollout_integer_parity_two_layers(name):
         for si, b in enumerate(seqs[:2]):
             ref = _oracle_state(gen, l, b, [[tok] for tok in io.evicted[si]])
             assert len(io.evicted[si]) == max(0, lens[b] - W)
+            assert np.abs(S[si] - ref).max() <= TOL_STATE
+    assert cache.status() == 0
+    cache.close()
+    torch.cuda.empty_cache()
+
+
+def test_paper_policy_at_full_size_pinned_prompt_and_quarter_window_chunks():
+    """The policy of the paper's runs (Sec. 3.3 / 4.1) on the 7B-shaped workload at full size: the prompt stays
+    pinned, the rest of the window slides, a quarter of the window is evicted at once and folded by the
+    tensor-core encoder.  Two eviction bursts; outputs and states at sampled points, ring state everywhere."""
+    c = _workload("qwen7b")
+    L, B, W, Hq, Hkv, D = c["n_layers"], c["batch"], c["window"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"]
+    E = W // 4
+    torch.cuda.empty_cache()
+    gen, cache = _make_cache(c, L, evict_chunk=E)
+    assert cache.info()["tensor_core_encode"]
+    n_prompt = gen.lengths(64, 700).numpy()
+    p_max = int(n_prompt.max())
+    Kp = gen.generic(50, 0, (L, B, p_max, Hkv, D), 1.0)
+    Vp = gen.generic(51, 0, (L, B, p_max, Hkv, D), 1.0)
+    cache.prefill(-1, Kp, Vp, torch.as_tensor(n_prompt, dtype=torch.int32, device="cuda:0"), p_max)
+    rng = np.random.default_rng(5)
+    seqs = sorted({int(np.argmin(n_prompt)), int(np.argmax(n_prompt)), *rng.integers(0, B, 3).tolist()})
+    layers = sorted({0, L - 1, int(rng.integers(0, L))})
+    io = _IntOracle(seqs, W, E)
+    io.prefill(n_prompt)
+    first_full = W - int(n_prompt.max())            # the sequence with the longest prompt fills first
+    T = W - int(n_prompt.min()) + E + 3             # every sequence has evicted at least once, most of them twice
+    checks = {0, first_full - 1, first_full, first_full + 1, T - 1} | set(rng.integers(first_full, T, 5).tolist())
+    out = torch.zeros(L, B, Hq, D, dtype=cache.torch_dtype, device="cuda:0")
+    evicted_chunks = [[] for _ in seqs]
+    worst, n_points = 0.0, 0
+    for j in range(T):
+        q = gen.step_q(j)
+        k, v = gen.step_kv(j)
+        cache.decode_step(-1, q, k, v, out)
+        _, ev_t, _ = io.step(None)
+        for si, toks in enumerate(ev_t):
+            if toks:
+                evicted_chunks[si].append(toks)
+        if j in checks:
+            out_h = np64(out[layers][:, seqs])
+            for li, l in enumerate(layers):
+                for si, b in enumerate(seqs):
+                    n = int(n_prompt[b])
+                    # token index t < n is prompt row t; t >= n is the (t - n)-th decoded token of the stream
+                    Kd, Vd = gen.token_kv(l, b, [t - n for t in io.live(si)])
+                    Kl = np.concatenate([np64(Kp[l, b, :n]), np64(Kd)])
+                    Vl = np.concatenate([np64(Vp[l, b, :n]), np64(Vd)])
+                    ref, _ = attention_gqa(np64(gen.token_q(l, b, j)), Kl, Vl)
+                    worst = max(worst, np.abs(out_h[li, si] - ref).max())
+                    n_points += 1
+    assert n_points >= 40 and worst <= TOL_OUT["bf16"], worst
+    for l in range(L):
+        head, count, n_app = cache.get_ring(l)
+        assert np.array_equal(cache.get_pinned(l).cpu().numpy(), n_prompt)
+        assert np.array_equal(n_app.cpu().numpy(), n_prompt + T)
+        cap = W - n_prompt
+        jj = T - 1
+        want = np.where(jj < cap, jj + 1, cap - E + 1 + (jj - cap) % E)
+        assert np.array_equal(count.cpu().numpy(), want)
+    for l in layers[:2]:
+        S = np64(cache.get_state(l)[seqs])
+        for si, b in enumerate(seqs[:3]):
+            n = int(n_prompt[b])
+            chunks = [[t - n for t in toks] for toks in evicted_chunks[si]]
+            assert chunks and all(len(ch) == E for ch in chunks)
+            ref = _oracle_state(gen, l, b, chunks)
             assert np.abs(S[si] - ref).max() <= TOL_STATE
     assert cache.status() == 0
     cache.close()
