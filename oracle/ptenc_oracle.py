@@ -31,6 +31,9 @@ in the tests where the mathematics allows):
 * S_0 is not normalised (the initialisation formula carries no Normalize)
   -- parity unpinned.
 * no softmax and no scaling inside the encoder (Eq. (3) has neither);
+* Delta W = A S_e B with A [d_out, G] and B [r, d_in]; which projection of the model receives it
+  is not stated, so the update is applied to a projection given by the caller (d_in, d_out free)
+  -- parity unpinned for that choice, the arithmetic itself is pinned;
 * order inside a step: evict, append, attend; the live set never exceeds W;
 * eviction is FIFO by arrival and freed slots are reused FIFO;
 * pinned question tokens (Sec. 3.3, the sliding-window policy keeps the question; Sec. 4.1): a
@@ -133,6 +136,25 @@ def initial_state(Qa, Wk_a, Wv_a, k_g, v_g):
 def encode_update(S, Qa, Wk_a, Wv_a, K_e, V_e, mode=0):
     """S <- Normalize(S + S') with S' the context state of the evicted rows."""
     return normalize(np.asarray(S, F64) + context_state(Qa, Wk_a, Wv_a, K_e, V_e), mode)
+
+
+# ----------------------------------------------------------------------------------
+# Dynamic weight update (Sec. 3.3, Eq. (3) and the sentence after it: theta' = theta + Delta W)
+# ----------------------------------------------------------------------------------
+def lora_delta(A, S, Bm):
+    """Delta W = A S_e B.  A [d_out, G], S [G, r], Bm [r, d_in] -> [d_out, d_in]."""
+    return np.asarray(A, F64) @ np.asarray(S, F64) @ np.asarray(Bm, F64)
+
+
+def lora_apply(y, x, A, S, Bm):
+    """Output of a projection whose weight received Delta W, given the output y = W x of the unchanged weight:
+    y' = (W + Delta W) x = y + Delta W x, per sequence (each sequence has its own state).
+    y [B, d_out], x [B, d_in], S [B, G, r]."""
+    y = np.asarray(y, F64).copy()
+    x = np.asarray(x, F64)
+    for b in range(y.shape[0]):
+        y[b] = y[b] + lora_delta(A, S[b], Bm) @ x[b]
+    return y
 
 
 # ----------------------------------------------------------------------------------

@@ -479,13 +479,46 @@ def pin_prompt_rows_never_reach_the_encoder(mod):
         ra, rb = a.append_evict(0, x, x), b.append_evict(0, x, x)
         assert list(ra[0]) == list(rb[0]) and ra[1] == rb[1] and ra[2] == rb[2]
 
+# ---------------------------------------------------------------- dynamic weight update (Sec. 3.3)
+def pin_lora_update(mod):
+    """Delta W = A S B on a hand-worked integer case, in exact rational arithmetic, and through the identities
+    (W + Delta W) x = W x + A (S (B x)), linearity in S, S = 0 changes nothing."""
+    A = np.array([[1, 2], [0, -1], [3, 1]])             # d_out 3, G 2
+    S = np.array([[2, 0, 1], [-1, 1, 0]])               # G 2, r 3
+    Bm = np.array([[1, 0, 2, 0], [0, 1, 0, -1], [1, 1, 0, 0]])   # r 3, d_in 4
+    # S B = [[3,1,4,0],[-1,1,-2,-1]];  A (S B) = [[1,3,0,-2],[1,-1,2,1],[8,4,10,-1]]
+    assert np.array_equal(mod.lora_delta(A, S, Bm), np.array([[1, 3, 0, -2], [1, -1, 2, 1], [8, 4, 10, -1]]))
+    rng = np.random.default_rng(21)
+    d_out, G, r, d_in, B = 5, 3, 4, 6, 2
+    Ai, Si, Bi = rng.integers(-4, 5, (d_out, G)), rng.integers(-4, 5, (B, G, r)), rng.integers(-4, 5, (r, d_in))
+    xi, yi = rng.integers(-4, 5, (B, d_in)), rng.integers(-4, 5, (B, d_out))
+    got = mod.lora_apply(yi, xi, Ai, Si, Bi)
+    for b in range(B):
+        for i in range(d_out):
+            want = Fraction(int(yi[b, i]))
+            for g in range(G):
+                for j in range(r):
+                    for d in range(d_in):
+                        want += Fraction(int(Ai[i, g])) * int(Si[b, g, j]) * int(Bi[j, d]) * int(xi[b, d])
+            assert Fraction(float(got[b, i])) == want
+    Af, Sf, Bf = rng.standard_normal((d_out, G)), rng.standard_normal((B, G, r)), rng.standard_normal((r, d_in))
+    x, Wm = rng.standard_normal((B, d_in)), rng.standard_normal((d_out, d_in))
+    y = x @ Wm.T
+    full = np.stack([(Wm + mod.lora_delta(Af, Sf[b], Bf)) @ x[b] for b in range(B)])
+    np.testing.assert_allclose(mod.lora_apply(y, x, Af, Sf, Bf), full, atol=1e-12)
+    fact = np.stack([y[b] + Af @ (Sf[b] @ (Bf @ x[b])) for b in range(B)])
+    np.testing.assert_allclose(mod.lora_apply(y, x, Af, Sf, Bf), fact, atol=1e-12)
+    np.testing.assert_allclose(mod.lora_apply(y, x, Af, 0 * Sf, Bf), y, atol=0)
+    two = mod.lora_apply(y, x, Af, 2 * Sf, Bf) - y
+    np.testing.assert_allclose(two, 2 * (mod.lora_apply(y, x, Af, Sf, Bf) - y), atol=1e-12)
+
 
 PINS = [pin_ring_closed_form, pin_ring_vs_list_model, pin_attention_full_window_is_causal,
         pin_attention_sliding_window, pin_attention_chunked_window, pin_attention_window_one,
         pin_attention_special_cases, pin_attention_gqa_mapping, pin_encode_worked_example,
         pin_encode_exact_rational, pin_encode_identities, pin_encode_recurrence,
         pin_staged_rows_are_evicted_tokens, pin_prompt_is_pinned_and_window_slides_over_the_rest,
-        pin_prompt_rows_never_reach_the_encoder]
+        pin_prompt_rows_never_reach_the_encoder, pin_lora_update]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -530,6 +563,10 @@ MUTATIONS = {
     "chunk_exceeds_capacity": ("for _ in range(min(self.E, capacity)):", "for _ in range(self.E):"),
     "stale_v": ("c.V[s_new] = v_new[b]", "c.V[s_new] = k_new[b]"),
     "encode_ignores_disable": ("if not self.encode_enabled:\n            return", "if False:\n            return"),
+    "lora_transposed_state": ("return np.asarray(A, F64) @ np.asarray(S, F64) @ np.asarray(Bm, F64)",
+                              "return np.asarray(A, F64) @ np.asarray(S, F64).T @ np.asarray(Bm, F64)"),
+    "lora_replaces_output": ("y[b] = y[b] + lora_delta(A, S[b], Bm) @ x[b]", "y[b] = lora_delta(A, S[b], Bm) @ x[b]"),
+    "lora_shared_state": ("y[b] = y[b] + lora_delta(A, S[b], Bm) @ x[b]", "y[b] = y[b] + lora_delta(A, S[0], Bm) @ x[b]"),
     "lse_without_max": ("return o, smax + np.log(z)", "return o, np.log(z)"),
 }
 
