@@ -150,6 +150,16 @@ PTENC_API int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const 
 PTENC_API int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e,
                  const int32_t* n_evicted /*[B]*/, int32_t m_max, void* stream);
 
+/* Dynamic weight update (Sec. 3.3, Eq. (3) and the sentence after it): the state drives a low-rank change of a
+ * weight, Delta W = A S_e B, and decoding continues with theta' = theta + Delta W.  Given the output y = W x of the
+ * unchanged projection for the token each sequence is decoding, this adds the change for that sequence's current
+ * state: y[b,:] += A (S[b] (B x[b,:])); Delta W itself is never formed.  A [d_out, G], Bm [r, d_in], x [B, d_in],
+ * y [B, d_out] in/out (leading [L] when layer == -1), all in the storage dtype; accumulation in fp32.  Which
+ * projection of the model receives the update is the caller's choice (the paper does not say): d_in and d_out are
+ * free, d_in * sizeof(element) must be a multiple of 16.  Rows of inactive sequences are not touched. */
+PTENC_API int ptenc_lora_apply(ptenc_cache* c, int layer, const void* A, const void* Bm, const void* x, void* y,
+                               const uint8_t* active, int32_t d_in, int32_t d_out, void* stream);
+
 /* a4.  One whole decode step: ptenc_append_evict ; ptenc_encode(staged rows) ; ptenc_decode_attn, with
  * the same results as the three calls.  q, out [B, H_q, D]; k_new, v_new [B, H_kv, D] (leading [L] when
  * layer == -1). */

@@ -21,7 +21,7 @@ DTYPE_FP32, DTYPE_BF16 = 0, 1
 NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
-           "ptenc_set_encoder", "ptenc_prefill", "ptenc_get_pinned", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_decode_step",
+           "ptenc_set_encoder", "ptenc_prefill", "ptenc_get_pinned", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_lora_apply", "ptenc_decode_step",
            "ptenc_host_staging_bytes", "ptenc_decode_step_host",
            "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count", "ptenc_strerror"]
 
@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_append_evict.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.ptenc_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.ptenc_encode.argtypes = [vp, i32, vp, vp, vp, ctypes.c_int32, vp]
+    lib.ptenc_lora_apply.argtypes = [vp, i32, vp, vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, vp]
     lib.ptenc_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.ptenc_host_staging_bytes.argtypes = [vp, i32, ctypes.POINTER(u64)]
     lib.ptenc_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u64, vp]
@@ -180,6 +181,11 @@ class Cache:
     def encode(self, layer, K_e=None, V_e=None, n_evicted=None, m_max=0):
         _check(lib.ptenc_encode(self._h, layer, _ptr(K_e), _ptr(V_e), _ptr(n_evicted), int(m_max), _stream()),
                "ptenc_encode")
+
+    def lora_apply(self, layer, A, Bm, x, y, active=None):
+        """y += A (S (Bm x)) per sequence; A [.., d_out, G], Bm [.., r, d_in], x [.., B, d_in], y [.., B, d_out]."""
+        _check(lib.ptenc_lora_apply(self._h, layer, _ptr(A), _ptr(Bm), _ptr(x), _ptr(y), _ptr(active),
+                                    int(x.shape[-1]), int(y.shape[-1]), _stream()), "ptenc_lora_apply")
 
     def decode_step(self, layer, q, k_new, v_new, out, active=None):
         _check(lib.ptenc_decode_step(self._h, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(active), _ptr(out),

@@ -286,6 +286,19 @@ int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e, co
              ? PTENC_OK : PTENC_ECUDA;
 }
 
+int ptenc_lora_apply(ptenc_cache* c, int layer, const void* A, const void* Bm, const void* x, void* y,
+                     const uint8_t* active, int32_t d_in, int32_t d_out, void* stream) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  if (A == nullptr || Bm == nullptr || x == nullptr || y == nullptr || d_in < 1 || d_out < 1) return PTENC_EINVAL;
+  if (((size_t)d_in * c->dev.elt) % 16 != 0) return PTENC_ESHAPE;     // rows of B and x are read as 16-byte vectors
+  if (misaligned(A) || misaligned(Bm) || misaligned(x) || misaligned(y)) return PTENC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return ok(ptenc_launch_lora_apply(c, l0, nl, A, Bm, x, y, active, d_in, d_out, st), "lora_apply", st)
+             ? PTENC_OK : PTENC_ECUDA;
+}
+
 int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
                       const uint8_t* active, void* out, void* stream) {
   int l0, nl;

@@ -85,6 +85,9 @@ bool ptenc_step_e1_usable(const ptenc_cache* c, const void* Ke, int m_max);
 cudaError_t ptenc_launch_step_e1(ptenc_cache* c, int l0, int nl, bool append, const void* k_new, const void* v_new,
                                  const uint8_t* active, const void* Ke, const void* Ve, const int32_t* n_ev,
                                  int m_max, cudaStream_t st);
+// y += A (S (B x)) per sequence with the layer's current states (dynamic weight update, Sec. 3.3).
+cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* A, const void* Bm, const void* x,
+                                    void* y, const uint8_t* active, int d_in, int d_out, cudaStream_t st);
 // Chunk encoder on tcgen05 (bf16, rank 16/32/64, d_kv % 64 == 0): tensor maps at create time, launch per call.
 bool ptenc_encode_tc_prepare(ptenc_cache* c);
 cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,

@@ -384,3 +384,35 @@ def test_prefill_misuse_sets_the_status_word():
     p.cache.prefill(-1, Kp, Kp, n, 8)
     assert p.cache.status() == 2 and p.cache.get_pinned(0).tolist() == [0, 3, 0]
     p.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_dynamic_weight_update_from_the_running_state(dtype):
+    """y += A (S (B x)) with the state the rollout has produced so far, per sequence, against the oracle's
+    (W + A S B) x written out; masked rows untouched; all layers in one call and one layer alone."""
+    from oracle.ptenc_oracle import lora_apply
+    L, B, G, r, d_in, d_out = 2, 11, 16, 24, 328, 200
+    p = Pair(pt, n_layers=L, batch=B, n_q_heads=4, n_kv_heads=2, head_dim=64, window=12, evict_chunk=3, dtype=dtype,
+             seed=77, n_global=G, rank=r)
+    for t in range(30):
+        p.step(t)
+    A = p.gen.generic(60, 0, (L, d_out, G), G ** -0.5)
+    Bm = p.gen.generic(61, 0, (L, r, d_in), d_in ** -0.5)
+    x = p.gen.generic(62, 0, (L, B, d_in), 1.0)
+    y0 = p.gen.generic(63, 0, (L, B, d_out), 1.0)
+    active = torch.tensor([1, 1, 0, 1, 1, 1, 1, 0, 1, 1, 1], dtype=torch.uint8, device="cuda")
+    y = y0.clone()
+    p.cache.lora_apply(-1, A, Bm, x, y, active)
+    y1 = y0[1].clone()
+    p.cache.lora_apply(1, A[1], Bm[1], x[1], y1)
+    m = active.bool().cpu().numpy()
+    tol = 2e-2 if dtype == "bf16" else 2e-5
+    for l in range(L):
+        ref = lora_apply(np64(y0[l]), np64(x[l]), np64(A[l]), p.orc.S[l], np64(Bm[l]))
+        got = np64(y[l])
+        assert np.abs(got[m] - ref[m]).max() <= tol
+        assert np.array_equal(got[~m], np64(y0[l])[~m])
+        assert np.abs(ref - np64(y0[l])).max() > 0.05            # the update is not a no-op
+    assert np.abs(np64(y1) - lora_apply(np64(y0[1]), np64(x[1]), np64(A[1]), p.orc.S[1], np64(Bm[1]))).max() <= tol
+    assert p.cache.status() == 0
+    p.close()
