@@ -156,7 +156,7 @@ PTENC_API int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const voi
  * state: y[b,:] += A (S[b] (B x[b,:])); Delta W itself is never formed.  A [d_out, G], Bm [r, d_in], x [B, d_in],
  * y [B, d_out] in/out (leading [L] when layer == -1), all in the storage dtype; accumulation in fp32.  Which
  * projection of the model receives the update is the caller's choice (the paper does not say): d_in and d_out are
- * free, d_in * sizeof(element) must be a multiple of 16.  Rows of inactive sequences are not touched. */
+ * free, d_in * sizeof(element) must be a multiple of 16 and at most 8192 bytes (PTENC_ESHAPE otherwise).  Rows of inactive sequences are not touched. */
 PTENC_API int ptenc_lora_apply(ptenc_cache* c, int layer, const void* A, const void* Bm, const void* x, void* y,
                                const uint8_t* active, int32_t d_in, int32_t d_out, void* stream);
 

@@ -293,6 +293,7 @@ int ptenc_lora_apply(ptenc_cache* c, int layer, const void* A, const void* Bm, c
   if (rc != PTENC_OK) return rc;
   if (A == nullptr || Bm == nullptr || x == nullptr || y == nullptr || d_in < 1 || d_out < 1) return PTENC_EINVAL;
   if (((size_t)d_in * c->dev.elt) % 16 != 0) return PTENC_ESHAPE;     // rows of B and x are read as 16-byte vectors
+  if ((size_t)d_in * c->dev.elt > 8 * 1024) return PTENC_ESHAPE;       // eight input rows are staged in shared memory
   if (misaligned(A) || misaligned(Bm) || misaligned(x) || misaligned(y)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   return ok(ptenc_launch_lora_apply(c, l0, nl, A, Bm, x, y, active, d_in, d_out, st), "lora_apply", st)
