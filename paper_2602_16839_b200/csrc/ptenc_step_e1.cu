@@ -82,7 +82,6 @@ k_step_e1(PtencDev p, E1Args a) {
   const int b = b0 + warp;                           // this warp's sequence
   const size_t lb = (size_t)l * B + b;
   const size_t ob = (size_t)li * B + b;
-  const bool enc_on = p.encode_enabled && p.enc_set[l];
   const int vpr = d_kv >> 3;                         // 16-byte vectors per token row (all KV heads)
   const int gr = G * r;
   float* S = p.S + lb * gr;
@@ -90,11 +89,42 @@ k_step_e1(PtencDev p, E1Args a) {
   const int n_tiles = 2 * tiles_per_map;
   const int n_pairs = d_kv >> 5;                     // 32 k-values per pair of mma steps
 
-  // ---- pull what the later phases read into L2 now (128-byte lines; harmless when it turns out unused) -------------
+  // ---- everything that does not depend on the ring state is requested first, in one round trip: the ring state
+  //      itself, the arriving rows, the encoder flag; then Q_a and L2 prefetches of what the later phases read ----------
+  int rs_head = 0, rs_count = 0, rs_sink = 0, rs_act = 0;
+  long long rs_n = 0;
+  uint4 nk[2], nv[2];
+  const bool pre_new = APPEND && vpr <= 64 && b < B;           // arriving rows fit two vectors per lane
+  if (APPEND) {
+    if (lane == 0 && b < B) {
+      rs_act = (a.active == nullptr) ? 1 : (int)a.active[b];
+      rs_head = p.head[lb];
+      rs_count = p.count[lb];
+      rs_sink = p.n_sink[lb];
+      rs_n = p.n_app[lb];
+    }
+    if (pre_new) {
+      const int vph = p.D >> 3;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int v = lane + 32 * u;
+        if (v < vpr) {
+          const int h = v / vph, vv = v - h * vph;
+          const size_t src = ((ob * p.Hkv + h) * p.D) * 2 + (size_t)vv * 16;
+          nk[u] = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.k_new) + src);
+          nv[u] = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.v_new) + src);
+        }
+      }
+    }
+  }
+  const bool enc_on = p.encode_enabled && p.enc_set[l];
   if (enc_on) {
+    for (int i = tid; i < gr; i += E1_THREADS) {
+      const int gi = i / r;
+      qa[gi * (r + 1) + (i - gi * r)] = p.Qa[(size_t)l * gr + i];
+    }
     if (b < B)
       for (int i = lane; i * 32 < gr; i += 32) e1_prefetch_l2(S + i * 32);
-    for (int i = tid; i * 32 < gr; i += E1_THREADS) e1_prefetch_l2(p.Qa + (size_t)l * gr + i * 32);
     for (int item = warp; item < n_tiles * KS; item += E1_WARPS) {
       const int tile = item % n_tiles, ks = item / n_tiles;
       const int mat = tile >= tiles_per_map ? 1 : 0;
@@ -111,12 +141,11 @@ k_step_e1(PtencDev p, E1Args a) {
   int m = 0;
   if (APPEND) {
     int ev_slot = 0, new_slot = -1;
-    const bool act = (b < B) && (a.active == nullptr || a.active[b] != 0);
     if (lane == 0 && b < B) {
-      if (act) {
-        int head = p.head[lb], count = p.count[lb];
-        const long long n = p.n_app[lb];
-        const int ns = p.n_sink[lb];                 // pinned prompt entries; the ring runs over slots [ns, W)
+      if (rs_act != 0) {
+        int head = rs_head, count = rs_count;
+        const long long n = rs_n;
+        const int ns = rs_sink;                      // pinned prompt entries; the ring runs over slots [ns, W)
         const int cap = W - ns;
         if (ns < 0 || cap < 1 || head < 0 || head >= cap || count < 0 || count > cap) {
           atomicOr(p.status, PTENC_ST_BAD_INDEX);
@@ -163,9 +192,17 @@ k_step_e1(PtencDev p, E1Args a) {
       if (new_slot >= 0) {
         // the same lane read this address above when the ring was full, so the read precedes the write
         const size_t dst = (((lb * p.Hkv + h) * W + new_slot) * p.D) * 2 + (size_t)vv * 16;
-        const size_t src = ((ob * p.Hkv + h) * p.D) * 2 + (size_t)vv * 16;
-        *reinterpret_cast<uint4*>(p.K + dst) = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.k_new) + src);
-        *reinterpret_cast<uint4*>(p.V + dst) = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.v_new) + src);
+        if (pre_new) {
+          const int u = v >> 5;                      // v = lane + 32 u, u < 2
+          *reinterpret_cast<uint4*>(p.K + dst) = u == 0 ? nk[0] : nk[1];
+          *reinterpret_cast<uint4*>(p.V + dst) = u == 0 ? nv[0] : nv[1];
+        } else {
+          const size_t src = ((ob * p.Hkv + h) * p.D) * 2 + (size_t)vv * 16;
+          *reinterpret_cast<uint4*>(p.K + dst) =
+              *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.k_new) + src);
+          *reinterpret_cast<uint4*>(p.V + dst) =
+              *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(a.v_new) + src);
+        }
       }
     }
   } else {
@@ -190,11 +227,6 @@ k_step_e1(PtencDev p, E1Args a) {
 
   constexpr int NB = 32 / RJ;                        // state rows per batch: 32 registers per lane
   if (__syncthreads_or(mine ? 1 : 0) == 0) return;   // also orders phase A's shared-memory writes
-
-  for (int i = tid; i < gr; i += E1_THREADS) {
-    const int gi = i / r;
-    qa[gi * (r + 1) + (i - gi * r)] = p.Qa[(size_t)l * gr + i];
-  }
 
   // ---- k_a = X_k W^a_K^T, v_a = X_v W^a_V^T : 2r/8 column tiles of 8, each split KS ways along d_kv ------------------
   {
