@@ -33,7 +33,7 @@ METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0026   # (dram read + write) / algorithmic, ncu, see profiles/
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0028   # (dram read + write) / algorithmic, ncu, see profiles/
 
 
 def workload_cfg(name: str) -> dict:
@@ -345,7 +345,7 @@ def run_gpu(args, c: dict):
         bm["attn"] /= K                                          # per launch / per step averages from here on
         bm["step"] /= K
         # DRAM bytes per algorithmic byte of the attention kernel, from the ncu capture summarised in
-        # profiles/attn_bf16_ncu_full_stress-w2048-b16.md (a smaller batch of the same shape; traffic grows in
+        # profiles/attn_bf16_and_step_e1_ncu_full_stress-w2048-b16.md (a smaller batch of the same shape; traffic grows in
         # proportion to the tiles processed), scaled to this launch.
         traffic = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE * bm["attn"] if c["dtype"] == "bf16" else None
         bm.pop("attn_per_step")
