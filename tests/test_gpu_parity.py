@@ -386,12 +386,13 @@ def test_prefill_misuse_sets_the_status_word():
     p.close()
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
-def test_dynamic_weight_update_from_the_running_state(dtype):
+@pytest.mark.parametrize("dtype,G,r,d_in,d_out", [("bf16", 16, 24, 328, 200), ("fp32", 16, 24, 328, 200),
+                                                  ("bf16", 32, 32, 352, 200), ("bf16", 64, 16, 1024, 520)])
+def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out):
     """y += A (S (B x)) with the state the rollout has produced so far, per sequence, against the oracle's
     (W + A S B) x written out; masked rows untouched; all layers in one call and one layer alone."""
     from oracle.ptenc_oracle import lora_apply
-    L, B, G, r, d_in, d_out = 2, 11, 16, 24, 328, 200
+    L, B = 2, 11      # the last two shape sets take the tensor-core kernel, the first two the shape-generic one
     p = Pair(pt, n_layers=L, batch=B, n_q_heads=4, n_kv_heads=2, head_dim=64, window=12, evict_chunk=3, dtype=dtype,
              seed=77, n_global=G, rank=r)
     for t in range(30):
