@@ -148,7 +148,7 @@ class ClockSampler:
 
 
 # ======================================================================================== CPU oracle legs
-def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1):
+def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, n_prompt: int = 0):
     """Times the CPU oracle, as it stands, on 1 layer x n_seq sequences at the full window.
     Returns (seconds per sampled step, threads used)."""
     from oracle.ptenc_oracle import OracleCache
@@ -163,7 +163,11 @@ def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1):
     for t in range(4):
         k, v = gen.step_kv(t)
         pool.append((gen.step_q(t)[0].double().numpy(), k[0].double().numpy(), v[0].double().numpy()))
-    for t in range(c["window"]):                      # fill (not timed)
+    if n_prompt > 0:                                   # pinned prompt, as on the GPU side
+        Kp = gen.generic(50, 0, (1, n_seq, n_prompt, c["n_kv_heads"], c["head_dim"]), 1.0)[0].double().numpy()
+        Vp = gen.generic(51, 0, (1, n_seq, n_prompt, c["n_kv_heads"], c["head_dim"]), 1.0)[0].double().numpy()
+        orc.prefill(0, Kp, Vp, [n_prompt] * n_seq)
+    for t in range(c["window"] - n_prompt):                  # fill (not timed)
         _, k, v = pool[t % 4]
         orc.append_evict(0, k, v)
     for t in range(warm):
@@ -181,7 +185,7 @@ def run_reference(args, c: dict):
     if rank_env()[0] != 0:
         return
     n_seq = 8 if c["batch"] >= 8 else c["batch"]
-    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup), E=args.evict_chunk)
+    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup), E=args.evict_chunk, n_prompt=args.prompt_len)
     value = n_seq / (sec * c["n_layers"])
     sample = (f"1 of {c['n_layers']} layers x {n_seq} of {c['batch']} sequences per step at window {c['window']} "
               f"(full, evicting); tokens/s = {n_seq} / (step time x {c['n_layers']} layers)")
@@ -370,7 +374,7 @@ def run_gpu(args, c: dict):
         }
         if world == 1 and not args.no_cpu_baseline:
             n_seq, n_steps = min(8, B), args.cpu_steps
-            sec, cores = oracle_sample(c, n_seq, n_steps, E=E)
+            sec, cores = oracle_sample(c, n_seq, n_steps, E=E, n_prompt=P)
             line["cpu_baseline"] = {
                 "value": n_seq / (sec * L), "unit": UNIT, "cores": cores, "kind": "oracle",
                 "sample": (f"oracle decode_step on 1 of {L} layers x {n_seq} of {B} sequences x {n_steps} steps at "

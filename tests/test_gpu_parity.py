@@ -417,3 +417,26 @@ def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out):
     assert np.abs(np64(y1) - lora_apply(np64(y0[1]), np64(x[1]), np64(A[1]), p.orc.S[1], np64(Bm[1]))).max() <= tol
     assert p.cache.status() == 0
     p.close()
+
+
+@pytest.mark.parametrize("W,E,prompts", [(150, 1, [0, 70, 149]), (300, 75, [64, 0, 130])])
+def test_head_dim_64_tensor_core_attention_with_pinned_prompt(W, E, prompts):
+    """The D = 64 variant of the TMA attention kernel (64-token tiles), several tiles, pinned entries that end inside
+    a tile, group size 7."""
+    p = Pair(pt, n_layers=2, batch=3, n_q_heads=14, n_kv_heads=2, head_dim=64, window=W, evict_chunk=E, dtype="bf16",
+             seed=W + 1, n_global=16, rank=16)
+    assert p.cache.info()["tensor_core_attn"]
+    p.prefill(prompts, max(prompts))
+    for t in range(W + 2 * E + 30):
+        if t % 5 == 0 or t > W - 3:
+            p.step(t)
+        else:
+            q = p.gen.step_q(t)
+            k, v = p.gen.step_kv(t)
+            p.cache.decode_step(-1, q, k, v, p.out)
+            for l in range(p.L):
+                p.orc.append_evict(l, np64(k[l]), np64(v[l]))
+                p.orc.encode(l)
+    p.check_ring(); p.check_state()
+    assert p.cache.status() == 0
+    p.close()
