@@ -169,12 +169,17 @@ PTENC_API int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const 
 /* a4 with HOST buffers: the same step as ptenc_decode_step, with q, k_new, v_new, active read from host
  * memory and out written to host memory.  The call enqueues the host-to-device copies into `dev_staging`
  * (device, 256-byte aligned, at least ptenc_host_staging_bytes), the step, and the device-to-host copy of out,
- * and returns without synchronising: synchronise `stream` before reading out_host or reusing the host inputs.
+ * and returns without synchronising: synchronise `stream` before reading out_host or reusing the host buffers.
  * To overlap the transfers with the kernels the copies run on two internal copy streams (host objects made on
- * the first call; no device memory) that are forked from `stream` and joined back into it before the call
- * returns, so everything stays ordered on `stream` for the caller; with layer = -1 the queries and outputs move
- * in groups of layers and each group's attention is its own launch.  Host buffers should be page-locked for the
- * copies to be asynchronous.  active_host may be NULL. */
+ * the first call; no device memory); the kernels run on `stream`, and `stream` is made to wait for the last
+ * device-to-host copy before the call returns, so a later synchronise of `stream` covers everything.  With
+ * layer = -1 the queries and outputs move in groups of layers and each group's attention is its own launch.
+ * The staging buffer has two halves which consecutive calls use in turn, so that the uploads of one step can run
+ * while the kernels of the step before are still busy.  Consequence for ordering: the host input buffers must hold
+ * their values when the call is made (written by the CPU, or by work that has already completed); except for the
+ * first call on a staging buffer, the uploads do not wait for earlier work on `stream`.  The staging buffer must
+ * not be touched by anything else between calls.  Host buffers should be page-locked for the copies to be
+ * asynchronous.  active_host may be NULL. */
 PTENC_API int ptenc_host_staging_bytes(ptenc_cache* c, int layer, size_t* bytes /*host, out*/);
 PTENC_API int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const void* k_new_host,
                                      const void* v_new_host, const uint8_t* active_host, void* out_host,

@@ -111,14 +111,14 @@ bool ensure_host_pipeline(ptenc_cache* c) {
   bool good = cudaStreamCreateWithFlags(&c->st_in, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&c->st_out, cudaStreamNonBlocking) == cudaSuccess;
   auto mk = [&](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
-  mk(&c->ev_start); mk(&c->ev_kv); mk(&c->ev_done);
+  mk(&c->ev_start); mk(&c->ev_kv); mk(&c->ev_done); mk(&c->ev_half[0]); mk(&c->ev_half[1]);
   for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) { mk(&c->ev_q[i]); mk(&c->ev_o[i]); }
   return good;
 }
 
 void release_host_pipeline(ptenc_cache* c) {
   auto rm = [](cudaEvent_t& e) { if (e != nullptr) { cudaEventDestroy(e); e = nullptr; } };
-  rm(c->ev_start); rm(c->ev_kv); rm(c->ev_done);
+  rm(c->ev_start); rm(c->ev_kv); rm(c->ev_done); rm(c->ev_half[0]); rm(c->ev_half[1]);
   for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) { rm(c->ev_q[i]); rm(c->ev_o[i]); }
   if (c->st_in != nullptr) { cudaStreamDestroy(c->st_in); c->st_in = nullptr; }
   if (c->st_out != nullptr) { cudaStreamDestroy(c->st_out); c->st_out = nullptr; }
@@ -163,7 +163,10 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   c->attn_grid = 0;
   c->ev_attn_begin = c->ev_attn_end = nullptr;
   c->st_in = c->st_out = nullptr;
-  c->ev_start = c->ev_kv = c->ev_done = nullptr;
+  c->ev_start = c->ev_kv = c->ev_done = c->ev_half[0] = c->ev_half[1] = nullptr;
+  c->host_staging_ptr = nullptr;
+  c->host_staging_size = 0;
+  c->host_flip = 0;
   for (int i = 0; i < ptenc_cache::HOST_GROUPS_MAX; ++i) c->ev_q[i] = c->ev_o[i] = nullptr;
 
   PtencDev& d = c->dev;
@@ -347,7 +350,7 @@ int ptenc_host_staging_bytes(ptenc_cache* c, int layer, size_t* bytes) {
   int rc = check_layer(c, layer, &l0, &nl);
   if (rc != PTENC_OK) return rc;
   if (bytes == nullptr) return PTENC_EINVAL;
-  *bytes = host_staging(c, nl).total;
+  *bytes = 2 * host_staging(c, nl).total;          // two halves: consecutive steps alternate between them
   return PTENC_OK;
 }
 
@@ -362,23 +365,49 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
     return PTENC_EINVAL;
   if ((reinterpret_cast<uintptr_t>(dev_staging) & 255) != 0) return PTENC_EALIGN;
   const HostStaging h = host_staging(c, nl);
-  if (staging_bytes < h.total) return PTENC_EWORKSPACE;
+  const size_t half_bytes = (staging_bytes / 2) & ~(size_t)255;
+  if (half_bytes < h.total) return PTENC_EWORKSPACE;
   if (!ensure_host_pipeline(c)) return PTENC_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  char* sb = static_cast<char*>(dev_staging);
   const PtencDev& d = c->dev;
   auto good = [](cudaError_t e) { return e == cudaSuccess; };
 
-  // Transfers run on two copy streams forked from `stream` and joined back into it, so that for the caller the
-  // whole call is still ordered on `stream`.  Keys/values go first (the append needs them); the queries and the
-  // outputs move in groups of layers, each group's attention starting as soon as its queries have landed and its
-  // outputs leaving while the next group computes.
-  int ng = (nl + 3) / 4;
-  if (ng > ptenc_cache::HOST_GROUPS_MAX) ng = ptenc_cache::HOST_GROUPS_MAX;
-  if (ng < 1) ng = 1;
-  if (!good(cudaEventRecord(c->ev_start, st)) || !good(cudaStreamWaitEvent(c->st_in, c->ev_start, 0)) ||
-      !good(cudaStreamWaitEvent(c->st_out, c->ev_start, 0)))
+  // Transfers run on two copy streams and join `stream` before the call returns.  Keys/values go first (the append
+  // needs them); the queries and the outputs move in groups of layers, each group's attention starting as soon as
+  // its queries have landed and its outputs leaving while the next group computes.  Consecutive calls alternate
+  // between the two halves of the staging buffer, so the uploads of a step may start while the kernels of the step
+  // before are still running: they wait only for their half to be free.  The first call on a staging buffer (or
+  // after its size changed) is ordered after everything enqueued on `stream` so far.
+  // Layer groups, sized 4, 8, 16, ... from the last layer backwards: the outputs of a group leave while the next,
+  // smaller group computes, and only the last four layers' outputs are still to be copied when the kernels end.
+  int gb[ptenc_cache::HOST_GROUPS_MAX + 1];
+  int ng = 0;
+  {
+    int ends[ptenc_cache::HOST_GROUPS_MAX + 1];
+    int at = nl, size = 4, n = 0;
+    ends[n++] = nl;
+    while (at > 0 && n < ptenc_cache::HOST_GROUPS_MAX) {
+      at = at - size > 0 ? at - size : 0;
+      ends[n++] = at;
+      size *= 2;
+    }
+    ends[n - 1] = 0;                                   // the first group takes whatever is left
+    ng = n - 1;
+    for (int i = 0; i <= ng; ++i) gb[i] = ends[ng - i];
+  }
+  const bool fresh = c->host_staging_ptr != dev_staging || c->host_staging_size != staging_bytes;
+  c->host_staging_ptr = dev_staging;
+  c->host_staging_size = staging_bytes;
+  const int half = c->host_flip;
+  c->host_flip ^= 1;
+  char* sb = static_cast<char*>(dev_staging) + (size_t)half * half_bytes;
+  if (fresh) {
+    if (!good(cudaEventRecord(c->ev_start, st)) || !good(cudaStreamWaitEvent(c->st_in, c->ev_start, 0)) ||
+        !good(cudaStreamWaitEvent(c->st_out, c->ev_start, 0)))
+      return PTENC_ECUDA;
+  } else if (!good(cudaStreamWaitEvent(c->st_in, c->ev_half[half], 0))) {
     return PTENC_ECUDA;
+  }
   const uint8_t* act = nullptr;
   if (active_host != nullptr) {
     if (!good(cudaMemcpyAsync(sb + h.active, active_host, c->cfg.batch, cudaMemcpyHostToDevice, c->st_in)))
@@ -391,7 +420,7 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
     return PTENC_ECUDA;
   const size_t q_layer = (size_t)d.B * d.d_q * d.elt;
   for (int g = 0; g < ng; ++g) {
-    const int a0 = g * nl / ng, a1 = (g + 1) * nl / ng;
+    const int a0 = gb[g], a1 = gb[g + 1];
     if (!good(cudaMemcpyAsync(sb + h.q + a0 * q_layer, static_cast<const char*>(q_host) + a0 * q_layer,
                               (size_t)(a1 - a0) * q_layer, cudaMemcpyHostToDevice, c->st_in)) ||
         !good(cudaEventRecord(c->ev_q[g], c->st_in)))
@@ -413,7 +442,7 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
   }
   // a2 group by group
   for (int g = 0; g < ng; ++g) {
-    const int a0 = g * nl / ng, a1 = (g + 1) * nl / ng;
+    const int a0 = gb[g], a1 = gb[g + 1];
     if (!good(cudaStreamWaitEvent(st, c->ev_q[g], 0))) return PTENC_ECUDA;
     if (!ok(launch_attn(c, l0 + a0, a1 - a0, sb + h.q + a0 * q_layer, act, sb + h.out + a0 * q_layer, nullptr, st),
             "decode_step_host/attn", st))
@@ -423,7 +452,8 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
                               (size_t)(a1 - a0) * q_layer, cudaMemcpyDeviceToHost, c->st_out)))
       return PTENC_ECUDA;
   }
-  if (!good(cudaEventRecord(c->ev_done, c->st_out)) || !good(cudaStreamWaitEvent(st, c->ev_done, 0)))
+  if (!good(cudaEventRecord(c->ev_half[half], c->st_out)) || !good(cudaEventRecord(c->ev_done, c->st_out)) ||
+      !good(cudaStreamWaitEvent(st, c->ev_done, 0)))
     return PTENC_ECUDA;
   return PTENC_OK;
 }

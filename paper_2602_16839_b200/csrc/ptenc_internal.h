@@ -58,6 +58,10 @@ struct ptenc_cache {
   static constexpr int HOST_GROUPS_MAX = 8;
   cudaStream_t st_in, st_out;
   cudaEvent_t ev_start, ev_kv, ev_done, ev_q[HOST_GROUPS_MAX], ev_o[HOST_GROUPS_MAX];
+  cudaEvent_t ev_half[2];       // a half of the staging buffer is free again (its outputs have left for the host)
+  void* host_staging_ptr;       // staging buffer of the last host-buffer step, and its size
+  size_t host_staging_size;
+  int host_flip;                // half used by the next host-buffer step
   bool tc_encode;               // tensor-core chunk encoder usable for this shape
   CUtensorMap tmWk, tmWv;       // 2-D maps over the encoder weights: rows = L*r, cols = d_kv
   CUtensorMap tmStageK, tmStageV;   // 2-D maps over the staged evicted rows: rows = L*B*E, cols = d_kv

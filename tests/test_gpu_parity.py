@@ -440,3 +440,33 @@ def test_head_dim_64_tensor_core_attention_with_pinned_prompt(W, E, prompts):
     p.check_ring(); p.check_state()
     assert p.cache.status() == 0
     p.close()
+
+
+def test_host_buffer_steps_back_to_back_without_synchronising():
+    """Six host-buffer steps enqueued with no synchronisation in between (the uploads of a step overlap the kernels of
+    the step before, two staging halves in turn), each with its own host buffers: every output equals the device
+    path's."""
+    kw = dict(n_layers=6, batch=9, n_q_heads=8, n_kv_heads=2, head_dim=128, window=40, evict_chunk=1, dtype="bf16",
+              seed=61)
+    a, b = Pair(pt, **kw), Pair(pt, **kw)
+    for t in range(45):                                     # rings full, evicting
+        a.step(t); b.step(t, check=False)
+    staging = torch.empty(b.cache.host_staging_bytes(-1), dtype=torch.uint8, device="cuda")
+    steps = range(45, 51)
+    host_in, host_out, want = [], [], []
+    for t in steps:
+        q = b.gen.step_q(t)
+        k, v = b.gen.step_kv(t)
+        host_in.append(tuple(x.cpu().pin_memory() for x in (q, k, v)))
+        host_out.append(torch.zeros(a.out.shape, dtype=a.out.dtype).pin_memory())
+    torch.cuda.synchronize()
+    for i, t in enumerate(steps):
+        b.cache.decode_step_host(-1, *host_in[i], host_out[i], staging)
+    torch.cuda.synchronize()
+    for i, t in enumerate(steps):
+        a.step(t)
+        assert float((host_out[i].float() - a.out.cpu().float()).abs().max()) <= 4e-3
+    for l in range(6):
+        assert torch.equal(a.cache.get_state(l), b.cache.get_state(l))
+    assert b.cache.status() == 0
+    a.close(); b.close()
