@@ -26,7 +26,9 @@
  * - Return value: PTENC_OK or a negative error code.  Arguments are validated on the host before any
  *   launch; nothing is launched when an error is returned.  Device-side anomalies (a bounded wait that
  *   ran out, an index outside its range) never trap: they set a status word read by ptenc_cache_status.
- * - A handle may be used from one host thread and one stream at a time.
+ * - A handle may be used from one host thread and one stream at a time.  The device the cache was created on
+ *   (ptenc_config.device) must be the calling thread's current CUDA device when an entry point is called;
+ *   ptenc_cache_create makes it current.
  * - Storage dtype (ptenc_config.dtype) applies to q, k, v, out, the rings and the encoder weights;
  *   the state S, the latent queries Q_a, lse and all accumulation are fp32.
  */

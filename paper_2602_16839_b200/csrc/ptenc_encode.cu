@@ -192,12 +192,10 @@ template <typename T>
 cudaError_t launch_encode_t(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
                             const int32_t* n_ev, int m_max, int mode, cudaStream_t st) {
   const size_t smem = encode_smem(c->dev);
-  static bool attr_done[2] = {false, false};
-  const int ti = sizeof(T) == 4 ? 0 : 1;
-  if (!attr_done[ti] && smem > 48 * 1024) {
+  static bool attr_done[PTENC_MAX_DEVICES] = {};          // one per instantiation of this template
+  if (smem > 48 * 1024 && ptenc_first_use(attr_done, c->cfg.device)) {
     cudaError_t e = cudaFuncSetAttribute(k_encode_rows<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done[ti] = true;
   }
   const int grid = mode == 1 ? 1 : nl * c->cfg.batch;
   k_encode_rows<T><<<grid, ENC_THREADS, smem, st>>>(c->dev, l0, (const T*)Ke, (const T*)Ve, n_ev, m_max, mode);

@@ -427,12 +427,11 @@ template <int R>
 cudaError_t tc_launch(ptenc_cache* c, const CUtensorMap& tmK, const CUtensorMap& tmV, const TcArgs& a, int nl,
                       cudaStream_t st) {
   const size_t smem = TcSmem<R>::total(c->dev.G);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[PTENC_MAX_DEVICES] = {};
+  if (ptenc_first_use(attr_done, c->cfg.device)) {
     cudaError_t e = cudaFuncSetAttribute(k_encode_chunk_tc<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)TcSmem<R>::total(128));
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   k_encode_chunk_tc<R><<<nl * c->cfg.batch, TC_THREADS, smem, st>>>(c->dev, tmK, tmV, c->tmWk, c->tmWv, a);
   c->launches++;

@@ -100,6 +100,15 @@ cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* K
 // shape is not covered, in which case the generic kernel serves it.
 bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err);
 
+// Kernel attributes are per device: a launcher sets them the first time it runs on a device.
+constexpr int PTENC_MAX_DEVICES = 64;
+inline bool ptenc_first_use(bool (&done)[PTENC_MAX_DEVICES], int device) {
+  if (device < 0 || device >= PTENC_MAX_DEVICES) return true;     // unknown ordinal: set the attribute every time
+  if (done[device]) return false;
+  done[device] = true;
+  return true;
+}
+
 // ---- small device helpers --------------------------------------------------------------------------
 __device__ __forceinline__ float ptenc_to_float(float x) { return x; }
 __device__ __forceinline__ float ptenc_to_float(__nv_bfloat16 x) { return __bfloat162float(x); }

@@ -334,11 +334,10 @@ cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* 
   if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && (d_out & 7) == 0 &&
       lr_mma_smem(p.G, p.r, d_in) <= 200 * 1024) {
     const size_t smem_m = lr_mma_smem(p.G, p.r, d_in);
-    static bool attr_m = false;
-    if (!attr_m) {
+    static bool attr_m[PTENC_MAX_DEVICES] = {};
+    if (ptenc_first_use(attr_m, c->cfg.device)) {
       cudaError_t e = cudaFuncSetAttribute(k_lora_apply_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
-      attr_m = true;
     }
     const int nb = (p.B + LR_SEQ - 1) / LR_SEQ;
     k_lora_apply_mma<<<nl * nb, LR_THREADS, smem_m, st>>>(p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm,
@@ -351,13 +350,12 @@ cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* 
                                        (((size_t)LR_SEQ * p.G * (p.r + 1) + 3) & ~(size_t)3)) +
                       (size_t)LR_SEQ * d_in * p.elt;
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[PTENC_MAX_DEVICES] = {};
+  if (ptenc_first_use(attr_done, c->cfg.device)) {
     cudaError_t e = cudaFuncSetAttribute(k_lora_apply<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k_lora_apply<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   const int nblk = (p.B + LR_SEQ - 1) / LR_SEQ;
   if (c->cfg.dtype == PTENC_DTYPE_FP32)

@@ -333,12 +333,11 @@ template <bool APPEND, int RJ>
 cudaError_t e1_launch_t(ptenc_cache* c, int nl, const E1Args& a, cudaStream_t st) {
   const PtencDev& p = c->dev;
   const size_t smem = e1_smem_bytes(p.G, p.r, p.d_kv);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[PTENC_MAX_DEVICES] = {};
+  if (ptenc_first_use(attr_done, c->cfg.device)) {
     cudaError_t e = cudaFuncSetAttribute(k_step_e1<APPEND, RJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   const int nblk = (p.B + E1_SEQ - 1) / E1_SEQ;
   k_step_e1<APPEND, RJ><<<nl * nblk, E1_THREADS, smem, st>>>(p, a);
