@@ -321,7 +321,7 @@ def run_gpu(args, c: dict):
     hpool = [tuple(x.cpu().pin_memory() for x in p) for p in pool]
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
     staging = torch.empty(cache.host_staging_bytes(-1), dtype=torch.uint8, device=dev)
-    Ke = max(3, min(K, 100))
+    Ke = max(3, min(K, 100)) if E == 1 else E          # chunked eviction: one whole period of E steps
     for t in range(3):
         cache.decode_step_host(-1, *hpool[t % R], hout, staging)
     sync_all()
@@ -396,6 +396,8 @@ def main():
     ap.add_argument("--evict-chunk", type=int, default=1,
                     help="tokens evicted at once when a ring is full (1 = ring per step, the timed configuration; "
                          "window/4 is the setting of the paper's runs, Sec. 4.1)")
+    ap.add_argument("--n-global", type=int, default=0,
+                    help="number of state vectors G (0 = the workload's own, 32; the paper's ablation uses 16/32/48/64)")
     ap.add_argument("--prompt-len", type=int, default=0,
                     help="tokens of a pinned prompt per sequence (kept for the whole rollout; the window slides over "
                          "the remaining slots)")
@@ -403,6 +405,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     c = workload_cfg(args.workload)
+    if args.n_global > 0:
+        c["n_global"] = args.n_global
     if args.impl == "reference":
         run_reference(args, c)
         return

@@ -302,3 +302,74 @@ def test_paper_policy_at_full_size_pinned_prompt_and_quarter_window_chunks():
     assert cache.status() == 0
     cache.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("G", [16, 48, 64])
+@pytest.mark.parametrize("ratio", [0.05, 0.25])
+def test_ablation_grid_global_tokens_and_eviction_ratio(G, ratio):
+    """The paper's ablations as configurations (Sec. 4.3: number of global tokens 16/48/64; appendix: eviction ratios
+    5 % to 25 % of the window): 7B head shapes, window 1024, four layers, three eviction bursts."""
+    c = {**_workload("qwen7b"), "window": 1024, "batch": 16, "n_global": G}
+    L, B, W = 4, c["batch"], c["window"]
+    E = max(1, int(round(ratio * W)))
+    torch.cuda.empty_cache()
+    gen, cache = _make_cache(c, L, evict_chunk=E)
+    seqs = [0, 7, 15]
+    io = _IntOracle(seqs, W, E)
+    T = W + 2 * E + 2
+    out = torch.zeros(L, B, c["n_q_heads"], c["head_dim"], dtype=cache.torch_dtype, device="cuda:0")
+    chunks = [[] for _ in seqs]
+    worst = 0.0
+    for t in range(T):
+        k, v = gen.step_kv(t)
+        if t >= W - 1:
+            q = gen.step_q(t)
+            cache.decode_step(-1, q, k, v, out)
+        else:
+            cache.append_evict(-1, k, v)
+        _, ev_t, _ = io.step(None)
+        for si, toks in enumerate(ev_t):
+            if toks:
+                chunks[si].append(toks)
+        if t in (W - 1, W, W + E, T - 1):
+            out_h = np64(out[:, seqs])
+            for l in (0, L - 1):
+                for si, b in enumerate(seqs):
+                    worst = max(worst, np.abs(out_h[l, si] - _oracle_out(gen, l, b, t, io.live(si))).max())
+    assert worst <= TOL_OUT["bf16"], worst
+    for l in (0, L - 1):
+        S = np64(cache.get_state(l)[seqs])
+        assert S.shape == (3, G, 32)
+        for si, b in enumerate(seqs):
+            assert len(chunks[si]) == 3
+            assert np.abs(S[si] - _oracle_state(gen, l, b, chunks[si])).max() <= TOL_STATE
+    assert cache.status() == 0
+    cache.close()
+    torch.cuda.empty_cache()
+
+
+def test_endurance_65536_steps_under_a_1k_window():
+    """A 64K-token generation under a 1K window (the length the paper reports reaching, Sec. 4.3): one layer, every
+    step through the fused step; slots bit-exact over all 65536 steps, state and outputs against the oracle at the
+    end of 64512 evictions."""
+    c = {**_workload("qwen7b"), "window": 1024, "batch": 8}
+    W, B, T = 1024, 8, 65536
+    torch.cuda.empty_cache()
+    gen, cache = _make_cache(c, 1)
+    out = torch.zeros(1, B, c["n_q_heads"], c["head_dim"], dtype=cache.torch_dtype, device="cuda:0")
+    for t in range(T):
+        k, v = gen.step_kv(t)
+        q = gen.step_q(t)
+        cache.decode_step(-1, q, k, v, out)
+    head, count, n_app = cache.get_ring(0)
+    assert (n_app == T).all() and (count == W).all() and (head == T % W).all()
+    for b in (0, B - 1):
+        live = list(range(T - W, T))
+        ref = _oracle_out(gen, 0, b, T - 1, live)
+        assert np.abs(np64(out[0, b]) - ref).max() <= TOL_OUT["bf16"]
+    S = np64(cache.get_state(0)[[0]])
+    ref = _oracle_state(gen, 0, 0, [[tok] for tok in range(T - W)])
+    assert np.abs(S[0] - ref).max() <= TOL_STATE
+    assert cache.status() == 0
+    cache.close()
+    torch.cuda.empty_cache()
