@@ -504,27 +504,41 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       continue;
     }
 
-    for (int idx = tid; idx < 8 * D; idx += NCONS) {
-      const int r = idx / D, d = idx - r * D;
+    // NCONS / 8 threads per query-head row: the row's merge weights are computed once per thread
+    {
+      constexpr int TPR = NCONS / 8;
+      const int r = tid / TPR, d0 = tid - r * TPR;
       float mt = -INFINITY;
 #pragma unroll
       for (int w = 0; w < NW; ++w) mt = fmaxf(mt, mb_ml[w * 16 + r]);
-      float lt = 0.f, acc = 0.f;
+      float wg[NW];
+      float lt = 0.f;
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
         const float mw = mb_ml[w * 16 + r];
-        const float wg = (mw == -INFINITY) ? 0.f : ex2(mw - mt);
-        lt = fmaf(wg, mb_ml[w * 16 + 8 + r], lt);
-        acc = fmaf(wg, mb_acc[(w * 8 + r) * SM::ACC_STRIDE + d], acc);
+        wg[w] = (mw == -INFINITY) ? 0.f : ex2(mw - mt);
+        lt = fmaf(wg[w], mb_ml[w * 16 + 8 + r], lt);
       }
       if (whole) {
         if (r < g) {
-          out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
-          if (lse != nullptr && d == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
+#pragma unroll
+          for (int d = d0; d < D; d += TPR) {
+            float acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) acc = fmaf(wg[w], mb_acc[(w * 8 + r) * SM::ACC_STRIDE + d], acc);
+            out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
+          }
+          if (lse != nullptr && d0 == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
         }
       } else {
-        p.part_acc[((size_t)my_slot * 8 + r) * D + d] = acc;
-        if (d == 0) { p.part_ml[my_slot * 16 + r] = mt; p.part_ml[my_slot * 16 + 8 + r] = lt; }
+#pragma unroll
+        for (int d = d0; d < D; d += TPR) {
+          float acc = 0.f;
+#pragma unroll
+          for (int w = 0; w < NW; ++w) acc = fmaf(wg[w], mb_acc[(w * 8 + r) * SM::ACC_STRIDE + d], acc);
+          p.part_acc[((size_t)my_slot * 8 + r) * D + d] = acc;
+        }
+        if (d0 == 0) { p.part_ml[my_slot * 16 + r] = mt; p.part_ml[my_slot * 16 + 8 + r] = lt; }
       }
     }
 
