@@ -96,11 +96,12 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
 }
 // D(16x8) += A(16x16) B(16x8) with rows 8..15 of A identically zero: only c0/c1 (rows 0..7) are kept.
 __device__ __forceinline__ void mma_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  float z0, z1;
+  float z0, z1;                  // accumulators of the unused rows 8..15
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
       : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
       : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+  asm volatile("" ::"f"(z0), "f"(z1));      // dropped
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;

@@ -103,7 +103,7 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
   __syncthreads();
   // ---- w[s][g] = <S_s[g,:], u_s> ------------------------------------------------------------------------------------
   for (int idx = tid; idx < nseq * G; idx += LR_THREADS) {
-    const int s = idx / G, g = idx - s * G;
+    const int s = idx / G;
     const float* Srow = Ss + (size_t)idx * (r + 1);
     float a = 0.f;
     for (int j = 0; j < r; ++j) a = fmaf(Srow[j], u[s * r + j], a);
@@ -154,11 +154,12 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
 // both operands, which leaves the sums unchanged.  S u in between is fp32 FMA.
 // ---------------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void lr_mma_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  float z0, z1;
+  float z0, z1;                  // accumulators of the unused rows 8..15
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
       : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
       : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
+  asm volatile("" ::"f"(z0), "f"(z1));      // dropped
 }
 __device__ __forceinline__ void lr_cp_async16(void* smem_dst, const void* gsrc) {
   const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
