@@ -10,6 +10,10 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
+    # The package refuses to import without its CUDA library; build it first when the tree is fresh or stale
+    # (nvcc cross-compiles for sm_100a without a GPU).
+    import __graft_entry__
+    __graft_entry__.build()
 
 
 def pytest_collection_modifyitems(config, items):

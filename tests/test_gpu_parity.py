@@ -470,3 +470,18 @@ def test_host_buffer_steps_back_to_back_without_synchronising():
         assert torch.equal(a.cache.get_state(l), b.cache.get_state(l))
     assert b.cache.status() == 0
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("E", [1, 3])
+@pytest.mark.parametrize("G,r", [(5, 12), (3, 40), (128, 128)])
+def test_odd_state_shapes_take_the_right_encoder(G, r, E):
+    """Ranks that are not a multiple of 8 (shape-generic encoder), a rank of 40 (warp-mma kernel for E = 1, generic for
+    chunks), and the largest state (128 x 128: four values of a state row per lane)."""
+    p = Pair(pt, n_layers=2, batch=3, n_q_heads=4, n_kv_heads=2, head_dim=64, window=11, evict_chunk=E, dtype="bf16",
+             seed=G + r + E, n_global=G, rank=r)
+    for t in range(40):
+        p.step(t)
+    p.check_state()
+    p.check_ring()
+    assert p.cache.status() == 0
+    p.close()
