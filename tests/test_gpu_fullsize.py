@@ -173,7 +173,8 @@ def test_whole_rollout_integer_parity_two_layers(name):
     io = _IntOracle(seqs, W, 1)
     check_steps = {0, W - 1, W, W + 1, 2 * W - 1, 2 * W, T - 1, int(lens.min()) - 1, int(lens.min())}
     check_steps |= {j * W + d for j in range(2, T // W, max(1, T // W // 4)) for d in (-1, 0)}
-    check_steps |= set(rng.integers(0, T, 8).tolist())
+    check_steps |= {int(lens[b]) - 1 for b in seqs}                  # the last step of each sampled sequence
+    check_steps |= set(rng.integers(0, T, 40).tolist())              # >= 256 random (layer, sequence, step) points
     slot = torch.full((T, B), -9, dtype=torch.int32, device="cuda:0")
     first = torch.full((T, B), -9, dtype=torch.int64, device="cuda:0")
     nev = torch.full((T, B), -9, dtype=torch.int32, device="cuda:0")
@@ -207,7 +208,7 @@ def test_whole_rollout_integer_parity_two_layers(name):
             cache.append_evict(1, k[1], v[1], active)
             cache.encode(1)
     assert worst <= TOL_OUT[c["dtype"]], worst
-    assert n_points >= 32
+    assert n_points >= 256
     slot_h, first_h, nev_h = slot.cpu().numpy(), first.cpu().numpy(), nev.cpu().numpy()
     # sampled sequences against the oracle's deque / free list, every step
     for si, b in enumerate(seqs):
