@@ -144,124 +144,118 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// bf16 path on warp-level mma.  Eight sequences are the first eight rows of the 16-row A operand (rows 8..15 are
-// zero and their accumulators are dropped).  Both thin products against the weights run on the tensor cores so that
-// the arithmetic and the bf16 unpacking leave the issue slots to the loads:
-//   u = X B^T   : A fragments from the staged inputs (shared memory), B fragments straight from B in L2;
+// bf16 path on warp-level mma.  Sixteen sequences are the 16 rows of the A operand.  Both thin products against the
+// weights run on the tensor cores so that the arithmetic and the bf16 unpacking leave the issue slots to the loads:
+//   u = X B^T   : A fragments straight from the inputs, B fragments straight from B (both L2), the column tiles of u
+//                 and splits of d_in spread over the 16 warps;
 //   y += w A^T  : w = S u is fp32; it is split into two bf16 terms w_hi + w_lo so that nothing but the final
 //                 rounding of y is lost, and A's rows are the B operand, again straight from L2.
 // A lane's 8 consecutive contraction values feed two mma steps; the contraction index is permuted the same way on
-// both operands, which leaves the sums unchanged.  S u in between is fp32 FMA.
+// both operands, which leaves the sums unchanged.  S u in between is fp32 FMA, a warp per sequence.
 // ---------------------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void lr_mma_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  float z0, z1;                  // accumulators of the unused rows 8..15
+constexpr int LM_SEQ = 16;
+constexpr int LM_THREADS = 512;
+constexpr int LM_WARPS = LM_THREADS / 32;
+
+__device__ __forceinline__ void lr_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
-      : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
-  asm volatile("" ::"f"(z0), "f"(z1));      // dropped
-}
-__device__ __forceinline__ void lr_cp_async16(void* smem_dst, const void* gsrc) {
-  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t lr_pack(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-
-__host__ __device__ inline int lr_xstride(int d_in) {          // bytes; = 64 mod 128: conflict-free 16-byte A loads
-  const int raw = d_in * 2;
-  return raw + ((64 - raw % 128) + 128) % 128;
+__host__ __device__ inline int lm_k_split(int r) {
+  const int tiles = r >> 3;
+  return tiles < LM_WARPS ? LM_WARPS / tiles : 1;
 }
-__host__ __device__ inline size_t lr_mma_smem(int G, int r, int d_in) {
-  // u [KS][8][r] fp32 | w_hi, w_lo [8][G] bf16 | x [8][xstride]
-  return (size_t)LR_WARPS * 8 * r * 4 / ((r >> 3) < LR_WARPS ? (r >> 3) : LR_WARPS) + (size_t)2 * 8 * G * 2 + 16 +
-         (size_t)LR_SEQ * lr_xstride(d_in);
+__host__ __device__ inline size_t lr_mma_smem(int G, int r) {
+  // u [KS][16][r] fp32 | w_hi, w_lo [16][G] bf16
+  return (size_t)lm_k_split(r) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
 }
 
-__global__ void __launch_bounds__(LR_THREADS)
+__global__ void __launch_bounds__(LM_THREADS)
 k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ Bm,
                  const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                  const uint8_t* __restrict__ active, int d_in, int d_out) {
   extern __shared__ __align__(16) uint8_t lm_smem[];
   const int G = p.G, r = p.r, B = p.B;
   const int n_tiles = r >> 3;                                   // column tiles of u
-  const int KS = n_tiles < LR_WARPS ? LR_WARPS / n_tiles : 1;   // warps sharing a tile split d_in
-  float* u = reinterpret_cast<float*>(lm_smem);                 // [KS][8][r]
-  __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u + KS * 8 * r);   // [8][G]
-  __nv_bfloat16* w_lo = w_hi + 8 * G;
-  const int xstride = lr_xstride(d_in);
-  uint8_t* xs = reinterpret_cast<uint8_t*>(w_lo + 8 * G);
-  xs += (16 - (reinterpret_cast<uintptr_t>(xs) & 15)) & 15;
+  const int KS = lm_k_split(r);                                 // warps sharing a tile split d_in
+  float* u = reinterpret_cast<float*>(lm_smem);                 // [KS][16][r]
+  __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u + KS * LM_SEQ * r);   // [16][G]
+  __nv_bfloat16* w_lo = w_hi + LM_SEQ * G;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qrow = lane >> 2, qcol = lane & 3;
-  const int nblk = (B + LR_SEQ - 1) / LR_SEQ;
+  const int nblk = (B + LM_SEQ - 1) / LM_SEQ;
   const int li = blockIdx.x / nblk;
-  const int b0 = (blockIdx.x - li * nblk) * LR_SEQ;
+  const int b0 = (blockIdx.x - li * nblk) * LM_SEQ;
   const int l = l0 + li;
-  const int nseq = min(LR_SEQ, B - b0);
+  const int nseq = min(LM_SEQ, B - b0);
   const __nv_bfloat16* Bl = Bm + (size_t)li * r * d_in;
   const __nv_bfloat16* Al = A + (size_t)li * d_out * G;
   const __nv_bfloat16* xl = x + ((size_t)li * B + b0) * d_in;
   __nv_bfloat16* yl = y + ((size_t)li * B + b0) * d_out;
+  const bool lo_ok = qrow < nseq, hi_ok = qrow + 8 < nseq;      // the two sequences whose rows this lane touches
 
-  // ---- everything the later phases read is asked into L2 now (128-byte lines), so that their loads are L2 hits --------
+  // ---- what the later phases read is asked into L2 now (128-byte lines) -------------------------------------------------
   {
     const char* pS = reinterpret_cast<const char*>(p.S + ((size_t)l * B + b0) * G * r);
-    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * G * r * 4; o += (size_t)LR_THREADS * 128)
+    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * G * r * 4; o += (size_t)LM_THREADS * 128)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(pS + o));
-    for (int s = 0; s < nseq; ++s)
-      for (size_t o = (size_t)tid * 128; o < (size_t)d_out * 2; o += (size_t)LR_THREADS * 128)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(yl + (size_t)s * d_out) + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)r * d_in * 2; o += (size_t)LR_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Bl) + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)d_out * G * 2; o += (size_t)LR_THREADS * 128)
+    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * d_out * 2; o += (size_t)LM_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(yl) + o));
+    for (size_t o = (size_t)tid * 128; o < (size_t)d_out * G * 2; o += (size_t)LM_THREADS * 128)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Al) + o));
+    for (size_t o = (size_t)tid * 128; o < (size_t)r * d_in * 2; o += (size_t)LM_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Bl) + o));
+    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * d_in * 2; o += (size_t)LM_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(xl) + o));
   }
-  // ---- the block's input rows -> shared memory, all copies in flight at once; missing rows are zero -------------
-  const int vpr = d_in >> 3;
-  for (int idx = tid; idx < LR_SEQ * vpr; idx += LR_THREADS) {
-    const int s = idx / vpr, v = idx - s * vpr;
-    if (s < nseq) lr_cp_async16(xs + s * xstride + v * 16, xl + (size_t)s * d_in + (size_t)v * 8);
-    else *reinterpret_cast<uint4*>(xs + s * xstride + v * 16) = make_uint4(0u, 0u, 0u, 0u);
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  __syncthreads();
 
-  // ---- u = X B^T ---------------------------------------------------------------------------------------------------
+  // ---- u = X B^T -------------------------------------------------------------------------------------------------------
   {
-    const int n_pairs = d_in >> 5;
-    for (int item = warp; item < n_tiles * KS; item += LR_WARPS) {
+    const int n_pairs = d_in >> 5;                              // 32 contraction values per pair of mma steps
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    for (int item = warp; item < n_tiles * KS; item += LM_WARPS) {
       const int tile = item % n_tiles, ks = item / n_tiles;
       const int s_lo = ks * n_pairs / KS, s_hi = (ks + 1) * n_pairs / KS;
       const __nv_bfloat16* wrow = Bl + (size_t)(tile * 8 + qrow) * d_in + qcol * 8;
-      const uint8_t* xa = xs + qrow * xstride + qcol * 16;
-      float c0 = 0.f, c1 = 0.f;
-      for (int s0 = s_lo; s0 < s_hi; s0 += 8) {
-        uint4 bw[8];
+      const __nv_bfloat16* xlo = xl + (size_t)qrow * d_in + qcol * 8;
+      const __nv_bfloat16* xhi = xlo + (size_t)8 * d_in;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int s0 = s_lo; s0 < s_hi; s0 += 4) {
+        uint4 bw[4], al[4], ah[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          if (s0 + q < s_hi) bw[q] = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(s0 + q) * 32));
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 4; ++q) {
           if (s0 + q < s_hi) {
-            const uint4 lo = *reinterpret_cast<const uint4*>(xa + (s0 + q) * 64);
-            lr_mma_top(c0, c1, lo.x, lo.y, bw[q].x, bw[q].y);
-            lr_mma_top(c0, c1, lo.z, lo.w, bw[q].z, bw[q].w);
+            bw[q] = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(s0 + q) * 32));
+            al[q] = lo_ok ? __ldg(reinterpret_cast<const uint4*>(xlo + (size_t)(s0 + q) * 32)) : zero4;
+            ah[q] = hi_ok ? __ldg(reinterpret_cast<const uint4*>(xhi + (size_t)(s0 + q) * 32)) : zero4;
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (s0 + q < s_hi) {
+            lr_mma(c, al[q].x, ah[q].x, al[q].y, ah[q].y, bw[q].x, bw[q].y);
+            lr_mma(c, al[q].z, ah[q].z, al[q].w, ah[q].w, bw[q].z, bw[q].w);
           }
         }
       }
-      float* dst = u + ((size_t)ks * 8 + qrow) * r + tile * 8 + 2 * qcol;
-      dst[0] = c0;
-      dst[1] = c1;
+      float* dst = u + ((size_t)ks * LM_SEQ + qrow) * r + tile * 8 + 2 * qcol;
+      dst[0] = c[0];
+      dst[1] = c[1];
+      dst[8 * r] = c[2];
+      dst[8 * r + 1] = c[3];
     }
   }
   __syncthreads();
   // ---- w = S u (fp32), split into two bf16 terms: a warp per sequence, a lane per state row ---------------------------
-  for (int s = warp; s < LR_SEQ; s += LR_WARPS) {
+  for (int s = warp; s < LM_SEQ; s += LM_WARPS) {
     for (int g = lane; g < G; g += 32) {
       float acc = 0.f;
       if (s < nseq) {
@@ -272,11 +266,13 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             float t = u[(size_t)s * r + j + k];
-            for (int ks = 1; ks < KS; ++ks) t += u[((size_t)ks * 8 + s) * r + j + k];
+            for (int ks = 1; ks < KS; ++ks) t += u[((size_t)ks * LM_SEQ + s) * r + j + k];
             uu[k] = t;
           }
-          acc = fmaf(sv.x, uu[0], acc); acc = fmaf(sv.y, uu[1], acc);
-          acc = fmaf(sv.z, uu[2], acc); acc = fmaf(sv.w, uu[3], acc);
+          acc = fmaf(sv.x, uu[0], acc);
+          acc = fmaf(sv.y, uu[1], acc);
+          acc = fmaf(sv.z, uu[2], acc);
+          acc = fmaf(sv.w, uu[3], acc);
         }
       }
       const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
@@ -288,38 +284,55 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
   // ---- y += w A^T : column tiles of 8 outputs, four per iteration so that a row's 64 bytes of y move together ---------
   {
     const int kp = G >> 5;                                      // pairs of mma steps along G
-    const bool row_ok = qrow < nseq && (active == nullptr || active[b0 + qrow] != 0);
+    const bool wr_lo = lo_ok && (active == nullptr || active[b0 + qrow] != 0);
+    const bool wr_hi = hi_ok && (active == nullptr || active[b0 + qrow + 8] != 0);
     const int n_out_tiles = d_out >> 3;
-    for (int t0 = warp * 4; t0 < n_out_tiles; t0 += LR_WARPS * 4) {
+    // the w fragments of the first 32 state rows do not depend on the output tile
+    const uint4 wh_l = *reinterpret_cast<const uint4*>(w_hi + qrow * G + qcol * 8);
+    const uint4 wh_h = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + qcol * 8);
+    const uint4 wl_l = *reinterpret_cast<const uint4*>(w_lo + qrow * G + qcol * 8);
+    const uint4 wl_h = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + qcol * 8);
+    for (int t0 = warp * 4; t0 < n_out_tiles; t0 += LM_WARPS * 4) {
       uint4 aw[4];
-      uint32_t yo[4];
+      uint32_t yl4[4], yh4[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int i0 = (t0 + q) * 8;
         if (t0 + q < n_out_tiles) {
+          const int i0 = (t0 + q) * 8;
           aw[q] = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + qcol * 8));
-          yo[q] = row_ok ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
+          yl4[q] = wr_lo ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
+          yh4[q] = wr_hi ? *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) : 0u;
         }
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         if (t0 + q >= n_out_tiles) break;
         const int i0 = (t0 + q) * 8;
-        float c0 = 0.f, c1 = 0.f;
-        for (int pp = 0; pp < kp; ++pp) {
-          uint4 bw = aw[q];
-          if (pp > 0) bw = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + pp * 32 + qcol * 8));
-          const uint4 wh = *reinterpret_cast<const uint4*>(w_hi + qrow * G + pp * 32 + qcol * 8);
-          const uint4 wl = *reinterpret_cast<const uint4*>(w_lo + qrow * G + pp * 32 + qcol * 8);
-          lr_mma_top(c0, c1, wh.x, wh.y, bw.x, bw.y);
-          lr_mma_top(c0, c1, wh.z, wh.w, bw.z, bw.w);
-          lr_mma_top(c0, c1, wl.x, wl.y, bw.x, bw.y);
-          lr_mma_top(c0, c1, wl.z, wl.w, bw.z, bw.w);
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw[q].x, aw[q].y);
+        lr_mma(c, wh_l.z, wh_h.z, wh_l.w, wh_h.w, aw[q].z, aw[q].w);
+        lr_mma(c, wl_l.x, wl_h.x, wl_l.y, wl_h.y, aw[q].x, aw[q].y);
+        lr_mma(c, wl_l.z, wl_h.z, wl_l.w, wl_h.w, aw[q].z, aw[q].w);
+        for (int pp = 1; pp < kp; ++pp) {                       // more than 32 state rows
+          const uint4 bw = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + pp * 32 + qcol * 8));
+          const uint4 a_hl = *reinterpret_cast<const uint4*>(w_hi + qrow * G + pp * 32 + qcol * 8);
+          const uint4 a_hh = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + pp * 32 + qcol * 8);
+          const uint4 a_ll = *reinterpret_cast<const uint4*>(w_lo + qrow * G + pp * 32 + qcol * 8);
+          const uint4 a_lh = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + pp * 32 + qcol * 8);
+          lr_mma(c, a_hl.x, a_hh.x, a_hl.y, a_hh.y, bw.x, bw.y);
+          lr_mma(c, a_hl.z, a_hh.z, a_hl.w, a_hh.w, bw.z, bw.w);
+          lr_mma(c, a_ll.x, a_lh.x, a_ll.y, a_lh.y, bw.x, bw.y);
+          lr_mma(c, a_ll.z, a_lh.z, a_ll.w, a_lh.w, bw.z, bw.w);
         }
-        if (row_ok) {
-          const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yo[q]);
+        if (wr_lo) {
+          const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yl4[q]);
           *reinterpret_cast<uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) =
-              lr_pack(__low2float(old) + c0, __high2float(old) + c1);
+              lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
+        }
+        if (wr_hi) {
+          const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yh4[q]);
+          *reinterpret_cast<uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) =
+              lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
         }
       }
     }
@@ -333,17 +346,11 @@ cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* 
   const PtencDev& p = c->dev;
   // tensor-core path: bf16, r a multiple of 8, G and d_in multiples of 32, d_out a multiple of 8
   if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && (d_out & 7) == 0 &&
-      lr_mma_smem(p.G, p.r, d_in) <= 200 * 1024) {
-    const size_t smem_m = lr_mma_smem(p.G, p.r, d_in);
-    static bool attr_m[PTENC_MAX_DEVICES] = {};
-    if (ptenc_first_use(attr_m, c->cfg.device)) {
-      cudaError_t e = cudaFuncSetAttribute(k_lora_apply_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-      if (e != cudaSuccess) return e;
-    }
-    const int nb = (p.B + LR_SEQ - 1) / LR_SEQ;
-    k_lora_apply_mma<<<nl * nb, LR_THREADS, smem_m, st>>>(p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm,
-                                                           (const __nv_bfloat16*)x, (__nv_bfloat16*)y, active, d_in,
-                                                           d_out);
+      lr_mma_smem(p.G, p.r) <= 48 * 1024) {
+    const int nb = (p.B + LM_SEQ - 1) / LM_SEQ;
+    k_lora_apply_mma<<<nl * nb, LM_THREADS, lr_mma_smem(p.G, p.r), st>>>(
+        p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, active,
+        d_in, d_out);
     c->launches++;
     return cudaGetLastError();
   }
