@@ -335,6 +335,50 @@ def run_gpu(args, c: dict):
     h2d = sum(x.numel() * x.element_size() for x in hpool[0])
     d2h = hout.numel() * hout.element_size()
 
+    # ---- side measurements of the two kernels that the step average hides (rank 0, on request) -------------------------
+    extras = {}
+    if rank == 0 and args.extras:
+        def timed(fn, n=20, flush=None):
+            ts = []
+            for _ in range(n):
+                if flush is not None:
+                    flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ts.sort()
+            return ts[len(ts) // 2]
+        elt = 2 if c["dtype"] == "bf16" else 4
+        G, r, d_kv, d_q = c["n_global"], c["rank"], Hkv * D, Hq * D
+        if E > 1:
+            # the encoder's burst: every sequence folds a chunk of E staged rows (the rows staged by the last evicting
+            # step are folded again on each call; the arithmetic and the traffic are those of a real burst)
+            n_done = (W - P) + Wm + K + 3 + Ke                    # decoded tokens so far (fill, warm-up, both timed loops)
+            t = n_done
+            while not evicts_at(t, W, E, P):
+                t += 1
+            for i in range(n_done, t + 1):                        # run on to the next evicting step
+                cache.append_evict(-1, pool[i % R][1], pool[i % R][2])
+            Ee = min(E, W - P)
+            ms = timed(lambda: cache.encode(-1))
+            by = L * B * (2 * Ee * d_kv * elt + 2 * G * r * 4)
+            fl = L * B * Ee * (4 * d_kv * r + 4 * r * r) + L * B * 2 * G * r * r
+            extras["encode_burst"] = {"ms": ms, "algorithmic_gbs": by / ms / 1e6, "tflops": fl / ms / 1e9,
+                                      "rows_per_sequence": Ee, "tensor_core_encode": cache.info()["tensor_core_encode"],
+                                      "how": "median of 20 ptenc_encode(layer=-1) calls on the staged chunk, CUDA events"}
+        # the dynamic weight update on a d_q x d_q projection, L2 flushed before each call
+        Am = gen.generic(60, 0, (L, d_q, G), G ** -0.5)
+        Bw = gen.generic(61, 0, (L, r, d_q), d_q ** -0.5)
+        xin = gen.generic(62, 0, (L, B, d_q), 1.0)
+        yio = gen.generic(63, 0, (L, B, d_q), 1.0)
+        flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+        ms = timed(lambda: cache.lora_apply(-1, Am, Bw, xin, yio), flush=flush)
+        by = L * (2 * G * d_q * elt + B * (3 * d_q * elt + G * r * 4))
+        extras["lora_apply"] = {"ms": ms, "algorithmic_gbs": by / ms / 1e6, "d_in": d_q, "d_out": d_q,
+                                "how": "median of 20 ptenc_lora_apply(layer=-1) calls, L2 flushed, CUDA events"}
+        del Am, Bw, xin, yio, flush
+
     # ---- max over ranks -------------------------------------------------------------------------------------
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
 
@@ -371,6 +415,7 @@ def run_gpu(args, c: dict):
             "hbm": {"step_algorithmic_gbs": step_gbs, "frac_of_8tbs": step_gbs / NOMINAL_HBM_GBS,
                     "frac_of_measured": step_gbs / peak, "algorithmic_bytes_per_step": bm["step"]},
             "device_status": status,
+            **({"extras": extras} if extras else {}),
         }
         if world == 1 and not args.no_cpu_baseline:
             n_seq, n_steps = min(8, B), args.cpu_steps
@@ -403,6 +448,9 @@ def main():
                          "the remaining slots)")
     ap.add_argument("--cpu-steps", type=int, default=128, help="steps of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the encoder's burst on a staged chunk (with --evict-chunk > 1) and the dynamic "
+                         "weight update, each alone")
     args = ap.parse_args()
     c = workload_cfg(args.workload)
     if args.n_global > 0:
