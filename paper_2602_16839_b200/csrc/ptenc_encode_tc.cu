@@ -6,7 +6,7 @@
 // contractions over d_kv (~ r flop per byte read): the one place on this path where the tensor cores are needed
 // to stay on the HBM roofline.
 //
-// One CTA per (layer, sequence) with evicted rows:
+// CTAs (two per SM) walk the (layer, sequence) units that have evicted rows; per CTA:
 //  * warp 0 (one lane): TMA producer.  Per pipeline item it loads a [rows x 64] slab of the evicted K (or V) rows
 //    and the matching [r x 64] slab of W^a_K (or W^a_V), both K-major with the 128-byte swizzle, into a stage
 //    guarded by full/empty mbarriers.  Plain loads, no multicast.
@@ -146,6 +146,7 @@ struct TcArgs {
   int staged;         // 1: m comes from n_staged and layers are absolute; 0: from n_ev, layers relative to l0
   const int32_t* n_ev;
   int m_max;
+  int nl;             // layers of the call
 };
 
 template <int R>
@@ -178,23 +179,28 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, G = p.G, d_kv = p.d_kv;
-  const int li = blockIdx.x / B, b = blockIdx.x - li * B;
-  const int l = a.l0 + li;
-  if (!p.encode_enabled || !p.enc_set[l]) return;
-  int m;
-  long long row0;
-  if (a.staged) {
-    m = p.n_staged[(size_t)l * B + b];
-    row0 = ((long long)l * B + b) * a.rows_per_seq;
-  } else {
-    m = a.n_ev[(size_t)li * B + b];
-    if (m > a.m_max) m = a.m_max;
-    row0 = ((long long)li * B + b) * a.rows_per_seq;
-  }
-  if (m <= 0) return;                                                // uniform over the CTA
-  const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
+  if (!p.encode_enabled) return;
+  const int n_units = a.nl * B;
   const int nkc = d_kv / TC_KC;
   const uint32_t tx_bytes = (uint32_t)(a.a_rows * TC_KC * 2 + SM::W_BYTES);
+  // The CTA walks the (layer, sequence) units u = blockIdx.x, blockIdx.x + gridDim.x, ...; every role takes the same
+  // walk and skips the same units (no encoder for the layer, nothing evicted).  Returns the unit's row count.
+  auto unit = [&](int u, int* l, int* b, long long* row0) -> int {
+    const int li = u / B;
+    *b = u - li * B;
+    *l = a.l0 + li;
+    if (!p.enc_set[*l]) return 0;
+    int m;
+    if (a.staged) {
+      m = p.n_staged[(size_t)(*l) * B + *b];
+      *row0 = ((long long)(*l) * B + *b) * a.rows_per_seq;
+    } else {
+      m = a.n_ev[(size_t)li * B + *b];
+      if (m > a.m_max) m = a.m_max;
+      *row0 = ((long long)li * B + *b) * a.rows_per_seq;
+    }
+    return m > 0 ? m : 0;
+  };
 
   if (tid == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { tc_mbar_init(bar_full + 8 * s, 1); tc_mbar_init(bar_empty + 8 * s, 1); }
@@ -209,7 +215,6 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
   if (a.a_rows < TC_M)
     for (int i = tid; i < TC_STAGES * SM::STAGE_BYTES / 16; i += TC_THREADS)
       reinterpret_cast<uint4*>(smem)[i] = make_uint4(0u, 0u, 0u, 0u);
-  for (int i = tid; i < G * R; i += TC_THREADS) qa_s[i] = p.Qa[(size_t)l * G * R + i];
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
     tc_tmem_alloc(tc_smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
@@ -225,17 +230,23 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
     if (lane == 0) {
       uint32_t n = 0;
       bool ok = true;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const int y = (int)(row0 + (long long)tile * a.a_rows);
-        for (int mat = 0; mat < 2 && ok; ++mat) {
-          for (int kc = 0; kc < nkc; ++kc, ++n) {
-            const uint32_t s = n % TC_STAGES;
-            if (!tc_mbar_wait(bar_empty + 8 * s, ((n / TC_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
-            const uint32_t dst = sbase + s * SM::STAGE_BYTES;
-            const uint32_t fb = bar_full + 8 * s;
-            tc_mbar_expect_tx(fb, tx_bytes);
-            tc_tma_load_2d(dst, mat ? &tmV : &tmK, kc * TC_KC, y, fb);
-            tc_tma_load_2d(dst + SM::A_BYTES, mat ? &tmWv : &tmWk, kc * TC_KC, l * R, fb);
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        int l, b;
+        long long row0;
+        const int m = unit(u, &l, &b, &row0);
+        const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
+        for (int tile = 0; tile < n_tiles && ok; ++tile) {
+          const int y = (int)(row0 + (long long)tile * a.a_rows);
+          for (int mat = 0; mat < 2 && ok; ++mat) {
+            for (int kc = 0; kc < nkc; ++kc, ++n) {
+              const uint32_t s = n % TC_STAGES;
+              if (!tc_mbar_wait(bar_empty + 8 * s, ((n / TC_STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+              const uint32_t dst = sbase + s * SM::STAGE_BYTES;
+              const uint32_t fb = bar_full + 8 * s;
+              tc_mbar_expect_tx(fb, tx_bytes);
+              tc_tma_load_2d(dst, mat ? &tmV : &tmK, kc * TC_KC, y, fb);
+              tc_tma_load_2d(dst + SM::A_BYTES, mat ? &tmWv : &tmWk, kc * TC_KC, l * R, fb);
+            }
           }
         }
       }
@@ -255,28 +266,34 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
     // ================================================================ MMA issuer
     if (lane == 0) {
       constexpr uint32_t IDESC = tc_idesc(R);
-      uint32_t n = 0;
+      uint32_t n = 0, gt = 0;                           // pipeline items and 128-token tiles issued so far
       bool ok = true;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const uint32_t bf = tile & 1;
-        if (!tc_mbar_wait(bar_tempty + 8 * bf, ((tile >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        for (int mat = 0; mat < 2 && ok; ++mat) {
-          const uint32_t d_tmem = tmem_base + bf * 2 * R + mat * R;
-          for (int kc = 0; kc < nkc; ++kc, ++n) {
-            const uint32_t s = n % TC_STAGES;
-            if (!tc_mbar_wait(bar_full + 8 * s, (n / TC_STAGES) & 1, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t a_addr = sbase + s * SM::STAGE_BYTES;
-            const uint32_t w_addr = a_addr + SM::A_BYTES;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        int l, b;
+        long long row0;
+        const int m = unit(u, &l, &b, &row0);
+        const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
+        for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
+          const uint32_t bf = gt & 1;
+          if (!tc_mbar_wait(bar_tempty + 8 * bf, ((gt >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          for (int mat = 0; mat < 2 && ok; ++mat) {
+            const uint32_t d_tmem = tmem_base + bf * 2 * R + mat * R;
+            for (int kc = 0; kc < nkc; ++kc, ++n) {
+              const uint32_t s = n % TC_STAGES;
+              if (!tc_mbar_wait(bar_full + 8 * s, (n / TC_STAGES) & 1, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t a_addr = sbase + s * SM::STAGE_BYTES;
+              const uint32_t w_addr = a_addr + SM::A_BYTES;
 #pragma unroll
-            for (int k4 = 0; k4 < TC_KC / 16; ++k4)
-              tc_mma(d_tmem, tc_smem_desc(a_addr + 32 * k4), tc_smem_desc(w_addr + 32 * k4), IDESC,
-                     (kc > 0 || k4 > 0) ? 1u : 0u);
-            tc_commit(bar_empty + 8 * s);
+              for (int k4 = 0; k4 < TC_KC / 16; ++k4)
+                tc_mma(d_tmem, tc_smem_desc(a_addr + 32 * k4), tc_smem_desc(w_addr + 32 * k4), IDESC,
+                       (kc > 0 || k4 > 0) ? 1u : 0u);
+              tc_commit(bar_empty + 8 * s);
+            }
           }
+          if (ok) tc_commit(bar_tfull + 8 * bf);
         }
-        if (ok) tc_commit(bar_tfull + 8 * bf);
       }
       if (!ok) {
         atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
@@ -292,57 +309,68 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
     const int q = warp & 3;                             // TMEM lane quarter this warp may read
     const int row = 32 * q + lane;
     const int jm = et / TPJ, k0 = (et - jm * TPJ) * KPT;
-    float acc[KPT];
-#pragma unroll
-    for (int i = 0; i < KPT; ++i) acc[i] = 0.f;
-    bool ok = true;
-    for (int tile = 0; tile < n_tiles && ok; ++tile) {
-      const uint32_t bf = tile & 1;
-      // The four warps must agree on going on: the barriers below count all 128 threads.  Each thread reports its
-      // own wait, thread 0 adds the other roles' flag, and everybody reads the verdict after a barrier.
-      if (!tc_mbar_wait(bar_tfull + 8 * bf, (tile >> 1) & 1, abort_flag)) *epi_abort = 1;
-      if (et == 0 && *abort_flag != 0) *epi_abort = 1;
-      tc_epi_sync();
-      if (*epi_abort != 0) { ok = false; break; }
-      tc_fence_after();
-      float kr[R], vr[R];
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + bf * 2 * R;
-#pragma unroll
-      for (int c = 0; c < R; c += 16) {
-        tc_ld16(taddr + c, kr + c);
-        tc_ld16(taddr + R + c, vr + c);
-      }
-      tc_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * bf);
-      const bool valid = (row < a.a_rows) && (tile * a.a_rows + row < m);
-#pragma unroll
-      for (int j = 0; j < R; ++j) ka_s[row * (R + 1) + j] = valid ? kr[j] : 0.f;
-#pragma unroll
-      for (int j = 0; j < R; j += 4)
-        *reinterpret_cast<float4*>(va_s + row * R + j) =
-            valid ? make_float4(vr[j], vr[j + 1], vr[j + 2], vr[j + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
-      tc_epi_sync();
-      // M2[jm][k0 .. k0 + KPT) += sum over the tile's rows of k_a[row][jm] * v_a[row][k]
-      for (int rr = 0; rr < TC_M; ++rr) {
-        const float kj = ka_s[rr * (R + 1) + jm];
-#pragma unroll
-        for (int i = 0; i < KPT; ++i) acc[i] = fmaf(kj, va_s[rr * R + k0 + i], acc[i]);
-      }
-      tc_epi_sync();
-    }
-    if (!ok && lane == 0) { atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT); *abort_flag = 1; }
-    // every epilogue thread reaches these barriers, also after an abort (the state is then left untouched)
-#pragma unroll
-    for (int i = 0; i < KPT; ++i) m2_s[jm * R + k0 + i] = acc[i];
-    tc_epi_sync();
-    const bool good = (*abort_flag == 0);
-    // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ...
-    float* S = p.S + ((size_t)l * B + b) * G * R;
     const int ew = et >> 5;
-    float total = 0.f;
-    if (good) {
+    uint32_t gt = 0;                                    // 128-token tiles consumed so far
+    int cur_l = -1;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      int l, b;
+      long long row0;
+      const int m = unit(u, &l, &b, &row0);
+      if (m <= 0) continue;                             // uniform over the CTA
+      const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
+      // Q_a of the unit's layer (the previous unit's last reads of it are behind this barrier)
+      tc_epi_sync();
+      if (l != cur_l) {
+        for (int i = et; i < G * R; i += TC_EPI) qa_s[i] = p.Qa[(size_t)l * G * R + i];
+        cur_l = l;
+      }
+      float acc[KPT];
+#pragma unroll
+      for (int i = 0; i < KPT; ++i) acc[i] = 0.f;
+      for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
+        const uint32_t bf = gt & 1;
+        // The four warps must agree on going on: the barriers below count all 128 threads.  Each thread reports its
+        // own wait, thread 0 adds the other roles' flag, and everybody reads the verdict after a barrier.
+        if (!tc_mbar_wait(bar_tfull + 8 * bf, (gt >> 1) & 1, abort_flag)) *epi_abort = 1;
+        if (et == 0 && *abort_flag != 0) *epi_abort = 1;
+        tc_epi_sync();
+        if (*epi_abort != 0) { ok = false; break; }
+        tc_fence_after();
+        float kr[R], vr[R];
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + bf * 2 * R;
+#pragma unroll
+        for (int c = 0; c < R; c += 16) {
+          tc_ld16(taddr + c, kr + c);
+          tc_ld16(taddr + R + c, vr + c);
+        }
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * bf);
+        const bool valid = (row < a.a_rows) && (tile * a.a_rows + row < m);
+#pragma unroll
+        for (int j = 0; j < R; ++j) ka_s[row * (R + 1) + j] = valid ? kr[j] : 0.f;
+#pragma unroll
+        for (int j = 0; j < R; j += 4)
+          *reinterpret_cast<float4*>(va_s + row * R + j) =
+              valid ? make_float4(vr[j], vr[j + 1], vr[j + 2], vr[j + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        tc_epi_sync();
+        // M2[jm][k0 .. k0 + KPT) += sum over the tile's rows of k_a[row][jm] * v_a[row][k]
+        for (int rr = 0; rr < TC_M; ++rr) {
+          const float kj = ka_s[rr * (R + 1) + jm];
+#pragma unroll
+          for (int i = 0; i < KPT; ++i) acc[i] = fmaf(kj, va_s[rr * R + k0 + i], acc[i]);
+        }
+        tc_epi_sync();
+      }
+      if (!ok) break;                                   // uniform: the verdict was read after a barrier
+#pragma unroll
+      for (int i = 0; i < KPT; ++i) m2_s[jm * R + k0 + i] = acc[i];
+      tc_epi_sync();
+      // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ...
+      float* S = p.S + ((size_t)l * B + b) * G * R;
+      float total = 0.f;
       for (int gi = ew; gi < G; gi += 4) {
         float val[(R + 31) / 32];
         float ss = 0.f;
@@ -368,16 +396,16 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
           if (k < R) S[gi * R + k] = val[jj] * sc;
         }
       }
-    }
-    if (p.norm_mode == PTENC_NORM_FROBENIUS) {
-      if (lane == 0) frob[ew] = total;
-      tc_epi_sync();
-      if (good) {
+      if (p.norm_mode == PTENC_NORM_FROBENIUS) {
+        if (lane == 0) frob[ew] = total;
+        tc_epi_sync();
         const float sc = 1.f / fmaxf(sqrtf(frob[0] + frob[1] + frob[2] + frob[3]), 1e-12f);
         for (int gi = ew; gi < G; gi += 4)
           for (int k = lane; k < R; k += 32) S[gi * R + k] *= sc;      // each lane rescales what it stored
       }
     }
+    // after an abort the remaining units are left untouched
+    if (!ok && lane == 0) { atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT); *abort_flag = 1; }
   }
 
   tc_fence_before();
@@ -433,7 +461,11 @@ cudaError_t tc_launch(ptenc_cache* c, const CUtensorMap& tmK, const CUtensorMap&
                                          (int)TcSmem<R>::total(128));
     if (e != cudaSuccess) return e;
   }
-  k_encode_chunk_tc<R><<<nl * c->cfg.batch, TC_THREADS, smem, st>>>(c->dev, tmK, tmV, c->tmWk, c->tmWv, a);
+  // persistent: two CTAs per SM walk the (layer, sequence) units, so barriers and tensor memory are set up once per
+  // CTA and the loads of a unit's first tile overlap the epilogue of the unit before
+  int grid = nl * c->cfg.batch;
+  if (grid > 2 * c->sm_count) grid = 2 * c->sm_count;
+  k_encode_chunk_tc<R><<<grid, TC_THREADS, smem, st>>>(c->dev, tmK, tmV, c->tmWk, c->tmWv, a);
   c->launches++;
   return cudaGetLastError();
 }
@@ -466,6 +498,7 @@ cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* K
   TcArgs a;
   memset(&a, 0, sizeof(a));
   a.l0 = l0;
+  a.nl = nl;
   CUtensorMap tmK, tmV;
   if (Ke == nullptr) {
     a.staged = 1;
