@@ -201,6 +201,15 @@ def run_reference(args, c: dict):
     print(json.dumps(line), flush=True)
 
 
+def l2_note(c: dict) -> str:
+    elt = 2 if c["dtype"] == "bf16" else 4
+    ring = 2 * c["n_layers"] * c["batch"] * c["n_kv_heads"] * c["head_dim"] * c["window"] * elt
+    if ring > 4 * 126e6:
+        return f"K/V rings read per step ({ring / 2**30:.2f} GiB) exceed the 126 MB L2 by {ring / 126e6:.0f}x; no flush needed"
+    return (f"K/V rings ({ring / 2**20:.2f} MiB) fit the 126 MB L2 and are not flushed: this workload is latency-bound and "
+            "carries no roofline claim")
+
+
 def config_block(args, c: dict) -> dict:
     return {"workload": args.workload, "n_layers": c["n_layers"], "batch_per_gpu": c["batch"],
             "n_q_heads": c["n_q_heads"], "n_kv_heads": c["n_kv_heads"], "head_dim": c["head_dim"],
@@ -209,7 +218,7 @@ def config_block(args, c: dict) -> dict:
                       else f"steady state: rings between {c['window'] - args.evict_chunk + 1} and {c['window']} tokens, "
                            f"every {args.evict_chunk}-th step evicts and encodes {args.evict_chunk} tokens per sequence"),
             "launch_mode": "all layers per call (layer = -1)",
-            "l2": "K/V rings read per step exceed the 126 MB L2 by >100x; no flush needed",
+            "l2": l2_note(c),
             "parallelism": f"dp{args.gpus} (batch shards, no collective on the path)"}
 
 
@@ -316,6 +325,7 @@ def run_gpu(args, c: dict):
     attn_ms = [a.elapsed_time(b) for a, b in zip(ev_a, ev_b)]
     clocks = sampler.stop() if sampler else None
     status = cache.status()
+    cache_info = cache.info()
 
     # ---- end to end: host buffers in, host buffer out, through ptenc_decode_step_host ------------------------
     hpool = [tuple(x.cpu().pin_memory() for x in p) for p in pool]
@@ -407,7 +417,8 @@ def run_gpu(args, c: dict):
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / Ke, "steps": Ke,
                     "call": "ptenc_decode_step_host (pinned host q/k/v in, host out)"},
             "gpu_launches": launches,
-            "roofline": {"bound": "hbm", "kernel": "decode attention (k_attn_bf16)", "achieved": attn_gbs,
+            "roofline": {"bound": "hbm", "kernel": ("decode attention (k_attn_bf16)" if cache_info["tensor_core_attn"]
+                                                     else "decode attention (k_attn_generic)"), "achieved": attn_gbs,
                          "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
                          "frac": attn_gbs / peak, "frac_of_8tbs": attn_gbs / NOMINAL_HBM_GBS,
                          "traffic": traffic, "algorithmic_bytes_per_launch": bm["attn"],
