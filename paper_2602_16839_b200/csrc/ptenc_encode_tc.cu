@@ -202,6 +202,17 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
     return m > 0 ? m : 0;
   };
 
+  // Most steps of a chunked rollout evict nothing: look at this CTA's units first and leave before any set-up.
+  {
+    int any = 0;
+    for (int u = blockIdx.x + tid * gridDim.x; u < n_units; u += TC_THREADS * gridDim.x) {
+      int l, b;
+      long long row0;
+      any |= unit(u, &l, &b, &row0) > 0 ? 1 : 0;
+    }
+    if (__syncthreads_or(any) == 0) return;
+  }
+
   if (tid == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { tc_mbar_init(bar_full + 8 * s, 1); tc_mbar_init(bar_empty + 8 * s, 1); }
     for (int i = 0; i < 2; ++i) { tc_mbar_init(bar_tfull + 8 * i, 1); tc_mbar_init(bar_tempty + 8 * i, 4); }
