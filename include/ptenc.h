@@ -85,7 +85,7 @@ typedef struct {
 
 /* Bytes of device workspace a cache with this configuration needs.  Host only, launches nothing.
  * Layout (all inside the workspace): K and V rings [L][B][H_kv][W][D]; ring state head/count (int32)
- * and n_appended (int64) [L][B]; evicted-row staging [L][B][E][H_kv*D] for K and for V; state S
+ * and n_appended (int64) [L][B], pinned-entry counts (int32) [L][B]; evicted-row staging [L][B][E][H_kv*D] for K and for V; state S
  * [L][B][G][r] fp32; per layer Q_a [G][r] fp32 and copies of W^a_K, W^a_V; split-K partials; status. */
 PTENC_API int ptenc_workspace_bytes(const ptenc_config* cfg /*host*/, size_t* bytes /*host, out*/);
 
@@ -98,8 +98,9 @@ PTENC_API int ptenc_cache_create(const ptenc_config* cfg /*host*/, void* dev_wor
 /* Frees the host handle only. */
 PTENC_API int ptenc_cache_destroy(ptenc_cache* c);
 
-/* Empties the rings of the sequences with seq_mask[b] != 0 (NULL = all) in every layer and puts their
- * state back to the layer's initial state S_0 (zero when no encoder was set). */
+/* Empties the caches of the sequences with seq_mask[b] != 0 (NULL = all) in every layer (ring and pinned prompt
+ * entries) and puts their state back to the layer's initial state S_0 (zero when no encoder was set).  With
+ * seq_mask == NULL the device status word is cleared too. */
 PTENC_API int ptenc_cache_reset(ptenc_cache* c, const uint8_t* seq_mask /*[B], nullable*/, void* stream);
 
 /* Encoder set-up for one layer (Sec. 3.3): stores W^a_K, W^a_V, computes Q_a = q_g W^a_Q^T [G,r] and the
@@ -130,9 +131,10 @@ PTENC_API int ptenc_get_pinned(ptenc_cache* c, int layer, int32_t* n_pinned, voi
  * sequence already holds W tokens, its E oldest tokens are evicted first (FIFO): their K/V rows are
  * copied, oldest first and KV heads concatenated, to the staging area for ptenc_encode, and their slots
  * are freed in that order.  The token is then stored in the oldest free slot.  With FIFO reuse the slot
- * of the t-th token of a sequence is t mod W.  Optional outputs ([B] each, nullable): slot_out = slot
+ * of the t-th token of a sequence is t mod W (with a pinned prompt of n tokens: n + (t - n) mod (W - n), a full
+ * cache meaning W - n sliding tokens, and chunks of min(E, W - n)).  Optional outputs ([B] each, nullable): slot_out = slot
  * written (-1 inactive); evict_first_out = index of the oldest evicted token (-1 if none);
- * n_evicted_out = number of tokens evicted (0 or E). */
+ * n_evicted_out = number of tokens evicted (0 or the chunk size). */
 PTENC_API int ptenc_append_evict(ptenc_cache* c, int layer, const void* k_new, const void* v_new,
                        const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
                        int32_t* n_evicted_out, void* stream);
