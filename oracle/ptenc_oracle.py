@@ -187,6 +187,7 @@ class OracleCache:
         self.seqs = [[_Seq(window, n_kv_heads, head_dim) for _ in range(batch)] for _ in range(n_layers)]
         self.enc = [None] * n_layers        # (Qa, Wk_a, Wv_a)
         self.S = [None] * n_layers          # [B, G, r]
+        self.S0 = [None] * n_layers         # [G, r] initial state of the layer
         self.staged = [[None] * batch for _ in range(n_layers)]   # (K_e, V_e) of the last append
 
     # -- set-up ------------------------------------------------------------------------
@@ -194,7 +195,20 @@ class OracleCache:
         Qa = latent_queries(Wq_a, q_g)
         S0 = initial_state(Qa, Wk_a, Wv_a, k_g, v_g)
         self.enc[layer] = (Qa, np.asarray(Wk_a, F64), np.asarray(Wv_a, F64))
+        self.S0[layer] = S0
         self.S[layer] = np.repeat(S0[None], self.B, axis=0)
+
+    def reset(self, seq_mask=None):
+        """A finished sequence gives its place to a new one: empty cache (no pinned prompt, no tokens) and the
+        layer's initial state again, in every layer.  seq_mask None = every sequence."""
+        for layer in range(self.L):
+            for b in range(self.B):
+                if seq_mask is not None and not seq_mask[b]:
+                    continue
+                self.seqs[layer][b] = _Seq(self.W, self.Hkv, self.D)
+                self.staged[layer][b] = None
+                if self.S[layer] is not None:
+                    self.S[layer][b] = self.S0[layer]
 
     # -- prompt: pinned entries -----------------------------------------------------------
     def prefill(self, layer, K_p, V_p, n_prompt):

@@ -485,3 +485,28 @@ def test_odd_state_shapes_take_the_right_encoder(G, r, E):
     p.check_ring()
     assert p.cache.status() == 0
     p.close()
+
+
+@pytest.mark.parametrize("dtype,E", [("bf16", 1), ("bf16", 8), ("fp32", 1)])
+def test_sequences_finish_and_their_places_are_reused(dtype, E):
+    """A rollout batch in which sequences end at different times: a finished sequence is reset, a new prompt is
+    pinned in its place, and it decodes on beside the others (which are in the middle of their windows)."""
+    B, W = 6, 40
+    p = Pair(pt, n_layers=2, batch=B, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 64, window=W,
+             evict_chunk=E, dtype=dtype, seed=90 + E, n_global=16, rank=16)
+    p.prefill([5, 0, 12, 30, 0, 39], 39)
+    rng = np.random.default_rng(4)
+    for t in range(150):
+        if t in (37, 61, 90, 133):                          # some sequences finish; new ones take their places
+            done = (rng.random(B) < 0.4).astype(np.uint8)
+            done[t % B] = 1
+            p.cache.reset(torch.as_tensor(done, device="cuda"))
+            p.orc.reset(done)
+            n_new = np.where(done, rng.integers(0, W, B), 0)
+            p.prefill(n_new.tolist(), max(1, int(n_new.max())), tensor_id=70 + t)
+            p.check_ring()
+        p.step(t)
+    p.check_ring()
+    p.check_state()
+    assert p.cache.status() == 0
+    p.close()

@@ -512,13 +512,37 @@ def pin_lora_update(mod):
     two = mod.lora_apply(y, x, Af, 2 * Sf, Bf) - y
     np.testing.assert_allclose(two, 2 * (mod.lora_apply(y, x, Af, Sf, Bf) - y), atol=1e-12)
 
+def pin_reset_gives_a_fresh_sequence(mod):
+    """After a reset a sequence behaves exactly like one in a new cache (same slots, evictions, outputs, state),
+    and the sequences that were not reset are untouched."""
+    rng = np.random.default_rng(31)
+    kw = dict(n_q_heads=2, n_kv_heads=1, head_dim=4, window=5, evict_chunk=2, batch=2, n_global=3, rank=2)
+    a, fresh = _mk(mod, **kw), _mk(mod, **kw)
+    enc = dict(Wq_a=rng.standard_normal((2, 8)), Wk_a=rng.standard_normal((2, 4)), Wv_a=rng.standard_normal((2, 4)),
+               q_g=rng.standard_normal((3, 8)), k_g=rng.standard_normal((3, 4)), v_g=rng.standard_normal((3, 4)))
+    a.set_encoder(0, **enc)
+    fresh.set_encoder(0, **enc)
+    for t in range(9):
+        x = rng.standard_normal((2, 1, 4))
+        a.decode_step(0, rng.standard_normal((2, 2, 4)), x, x)
+    kept_S, kept_ring = a.S[0][1].copy(), [r[1] for r in a.ring(0)]
+    a.reset([1, 0])
+    assert [r[1] for r in a.ring(0)] == kept_ring and np.array_equal(a.S[0][1], kept_S)
+    assert [r[0] for r in a.ring(0)] == [0, 0, 0] and list(a.pinned_count(0)) == [0, 0]
+    for t in range(9):
+        q, x = rng.standard_normal((2, 2, 4)), rng.standard_normal((2, 1, 4))
+        oa, _, ra = a.decode_step(0, q, x, x, active=[1, 0])
+        of, _, rf = fresh.decode_step(0, q, x, x, active=[1, 0])
+        assert np.array_equal(oa[0], of[0]) and ra[0][0] == rf[0][0] and ra[1][0] == rf[1][0]
+        assert np.array_equal(a.S[0][0], fresh.S[0][0])
+
 
 PINS = [pin_ring_closed_form, pin_ring_vs_list_model, pin_attention_full_window_is_causal,
         pin_attention_sliding_window, pin_attention_chunked_window, pin_attention_window_one,
         pin_attention_special_cases, pin_attention_gqa_mapping, pin_encode_worked_example,
         pin_encode_exact_rational, pin_encode_identities, pin_encode_recurrence,
         pin_staged_rows_are_evicted_tokens, pin_prompt_is_pinned_and_window_slides_over_the_rest,
-        pin_prompt_rows_never_reach_the_encoder, pin_lora_update]
+        pin_prompt_rows_never_reach_the_encoder, pin_lora_update, pin_reset_gives_a_fresh_sequence]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
