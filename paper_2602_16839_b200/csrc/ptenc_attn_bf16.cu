@@ -39,6 +39,9 @@
 #ifndef PTENC_ATTN_CTAS_PER_SM
 #define PTENC_ATTN_CTAS_PER_SM 1
 #endif
+#ifndef PTENC_ATTN_TRY_WAIT
+#define PTENC_ATTN_TRY_WAIT 1        // park waiting threads (mbarrier.try_wait) instead of spinning on test_wait
+#endif
 #ifndef PTENC_ATTN_L2PROMO
 #define PTENC_ATTN_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
@@ -71,11 +74,25 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+#if PTENC_ATTN_TRY_WAIT
+  // try_wait lets the hardware park the thread (up to the hint, in ns) instead of spinning on test_wait
+  for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    if (ok) return true;
+  }
+  return false;
+#else
   for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
     if (mbar_test(bar, parity)) return true;
     if (i > 128) __nanosleep(128);
   }
   return false;
+#endif
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
