@@ -13,9 +13,11 @@
 //    multicast) into a ring of shared-memory stages guarded by full/empty mbarriers.
 //  * Each consumer warp owns whole tiles (tile n of the CTA goes to warp n mod NW, stage n mod STAGES; STAGES
 //    is a multiple of NW so a stage always has the same consumer warp and its full/empty barriers advance
-//    one phase per visit -- a warp can never be a phase ahead of a barrier it polls): S = Q K^T and O += P V
-//    run on warp-level bf16 mma (m16n8k16, fp32 accumulate) with the g query heads in the M rows, only to
-//    keep the FP32 pipes free; online softmax with quad shuffles; per-warp (m, l, O) partials.
+//    one phase per visit -- a warp can never be a phase ahead of a barrier it polls).  The two products run on
+//    warp-level bf16 mma (m16n8k16, fp32 accumulate) only to keep the FP32 pipes free, in transposed form so that
+//    all 16 rows of the mma carry data: S^T = K Q^T (rows = 16 tokens, columns = the g <= 8 query heads) and
+//    O^T += V^T P^T (rows = 16 head dims, columns = heads); P^T is turned from accumulator layout into a B
+//    fragment with movmatrix.  Online softmax per head, reduced over the lanes' token rows; per-warp (m, l, O).
 //  * Per unit the warps' partials are merged in shared memory (fp32).  A unit that is split between CTAs
 //    goes through fp32 partials in global scratch; the CTA that arrives last (atomic ticket) combines them.
 //    No CTA ever waits for another.
@@ -39,16 +41,13 @@
 #ifndef PTENC_ATTN_CTAS_PER_SM
 #define PTENC_ATTN_CTAS_PER_SM 1
 #endif
-#ifndef PTENC_ATTN_TRY_WAIT
-#define PTENC_ATTN_TRY_WAIT 1        // park waiting threads (mbarrier.try_wait) instead of spinning on test_wait
-#endif
 #ifndef PTENC_ATTN_L2PROMO
 #define PTENC_ATTN_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
 
 namespace {
 
-constexpr uint32_t WAIT_POLLS = 4000000;   // bounded wait: polls before giving up (~ a second)
+constexpr uint32_t WAIT_POLLS = 4000000;   // bounded wait: tries of up to a microsecond each before giving up
 
 // ------------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -63,19 +62,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok;
-}
-// Bounded wait.  Returns false when the limit ran out.
+// Bounded wait.  try_wait lets the hardware park the thread (up to the hint, in ns) instead of spinning on the
+// barrier; the loop bounds the total.  Returns false when the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-#if PTENC_ATTN_TRY_WAIT
-  // try_wait lets the hardware park the thread (up to the hint, in ns) instead of spinning on test_wait
   for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
     uint32_t ok;
     asm volatile(
@@ -86,13 +75,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (ok) return true;
   }
   return false;
-#else
-  for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
-    if (mbar_test(bar, parity)) return true;
-    if (i > 128) __nanosleep(128);
-  }
-  return false;
-#endif
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -111,14 +93,19 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-// D(16x8) += A(16x16) B(16x8) with rows 8..15 of A identically zero: only c0/c1 (rows 0..7) are kept.
-__device__ __forceinline__ void mma_top(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  float z0, z1;                  // accumulators of the unused rows 8..15
+// D(16x8) += A(16x16) B(16x8), all sixteen rows in use.
+__device__ __forceinline__ void mma_full(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
-      : "+f"(c0), "+f"(c1), "=f"(z0), "=f"(z1)
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.f));
-  asm volatile("" ::"f"(z0), "f"(z1));      // dropped
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Transposes an 8x8 matrix of 16-bit values held one row pair per lane across the warp.
+__device__ __forceinline__ uint32_t movm_t(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -182,8 +169,6 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
             __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
   using SM = Smem<D, TILE_N, NW, STAGES>;
-  constexpr int NT8 = TILE_N / 8;              // 8-token n-tiles of S
-  constexpr int KT16 = TILE_N / 16;            // 16-token k-steps of P V
   constexpr int NTHREADS = (NW + 1) * 32;
   constexpr int NCONS = NW * 32;
   constexpr int KSTEPS = D / 16;
@@ -390,12 +375,16 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       if (lane == 0) mbar_arrive(bar_qempty + 8 * ubuf);
     }
 
-    float m_run = -INFINITY, l_run = 0.f;
-    float o[D / 8][2];
+    // Transposed products, so that the 16 rows of the mma are always full: S^T = K Q^T (rows = tokens, columns = the
+    // query heads) and O^T += V^T P^T (rows = head dims, columns = heads).  A lane (qr, qc) then owns the two heads
+    // 2 qc and 2 qc + 1: their running maxima and sums, and the columns of O^T that belong to them.
+    constexpr int MT = TILE_N / 16;                // 16-token row tiles of S^T = k-steps of the second product
+    constexpr int DT = D / 16;                     // 16-dim row tiles of O^T
+    float m_run0 = -INFINITY, m_run1 = -INFINITY, l_run0 = 0.f, l_run1 = 0.f;
+    float oT[DT][4];
 #pragma unroll
-    for (int i = 0; i < D / 8; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; }
+    for (int i = 0; i < DT; ++i) { oT[i][0] = 0.f; oT[i][1] = 0.f; oT[i][2] = 0.f; oT[i][3] = 0.f; }
 
-    // tiles of this unit that fall to this warp: sequence numbers n + i with (n + i) % NW == warp
     int i0 = (int)((warp + NW - (n % NW)) % NW);
     for (int i = i0; i < n_mine; i += NW) {
       const uint32_t seq = n + i;
@@ -410,25 +399,23 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       const uint32_t kb = smem_base + s * SM::STAGE_BYTES;
       const uint32_t vb = kb + SM::K_BYTES;
 
-      // ---- S = Q K^T (8 heads x 64 tokens), fp32 ---------------------------------------------------------
-      float sc[NT8][2];
+      // ---- S^T = K Q^T: A = a 16-token x 16-dim block of K (ldmatrix), B = the Q fragments ----------------------
+      float sT[MT][4];
 #pragma unroll
-      for (int nt = 0; nt < NT8; ++nt) { sc[nt][0] = 0.f; sc[nt][1] = 0.f; }
+      for (int mt = 0; mt < MT; ++mt) { sT[mt][0] = 0.f; sT[mt][1] = 0.f; sT[mt][2] = 0.f; sT[mt][3] = 0.f; }
 #pragma unroll
-      for (int kp = 0; kp < KSTEPS / 2; ++kp) {
-        const int cidx = 4 * kp + (lane >> 3);               // 16-byte chunk of the row
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        const int cidx = 2 * ks + (lane >> 4);               // 16-byte chunk of the row
         const int hf = cidx >> 3, cc = cidx & 7;
 #pragma unroll
-        for (int nt = 0; nt < NT8; ++nt) {
-          const int row = 8 * nt + (lane & 7);
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), b0, b1, b2, b3);
-          mma_top(sc[nt][0], sc[nt][1], qa[2 * kp][0], qa[2 * kp][1], b0, b1);
-          mma_top(sc[nt][0], sc[nt][1], qa[2 * kp + 1][0], qa[2 * kp + 1][1], b2, b3);
+        for (int mt = 0; mt < MT; ++mt) {
+          const int row = 16 * mt + (lane & 7) + ((lane >> 3) & 1) * 8;
+          uint32_t a0, a1, a2, a3;
+          ldsm_x4(kb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), a0, a1, a2, a3);
+          mma_full(sT[mt], a0, a1, a2, a3, qa[ks][0], qa[ks][1]);
         }
       }
-      // ---- mask slots that hold no live token -------------------------------------------------------------
-      // live: a pinned entry (slot < sink), or a sliding slot whose distance from the head is below count
+      // ---- mask slots that hold no live token (rows qr and qr + 8 of each row tile) -------------------------------
       const int slot0 = j * TILE_N;
       bool full = false;
       if (slot0 + TILE_N <= sink) {
@@ -440,70 +427,93 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       }
       if (!full) {
 #pragma unroll
-        for (int nt = 0; nt < NT8; ++nt) {
+        for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
           for (int x = 0; x < 2; ++x) {
-            const int slot = slot0 + 8 * nt + 2 * qc + x;
+            const int slot = slot0 + 16 * mt + qr + 8 * x;
             int dd = slot - sink - head;
             if (dd < 0) dd += cap;
             const bool live = slot < sink || (slot < W && dd < count);
-            if (!live) sc[nt][x] = -INFINITY;
+            if (!live) { sT[mt][2 * x] = -INFINITY; sT[mt][2 * x + 1] = -INFINITY; }
           }
         }
       }
-      // ---- online softmax (base 2) ---------------------------------------------------------------------------
-      float mx = sc[0][0];
+      // ---- online softmax (base 2), two heads per lane, reduced over the eight token rows of the lanes ----------
+      float mx0 = sT[0][0], mx1 = sT[0][1];
 #pragma unroll
-      for (int nt = 0; nt < NT8; ++nt) { mx = fmaxf(mx, sc[nt][0]); mx = fmaxf(mx, sc[nt][1]); }
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(m_run, mx * sl2);
-      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // all-masked row: keep exp2 arguments finite
-      const float corr = ex2(m_run - m_use);
-      float psum = 0.f;
-      uint32_t pa[KT16][2];
-#pragma unroll
-      for (int kt = 0; kt < KT16; ++kt) {
-        const float p00 = ex2(fmaf(sc[2 * kt][0], sl2, -m_use));
-        const float p01 = ex2(fmaf(sc[2 * kt][1], sl2, -m_use));
-        const float p10 = ex2(fmaf(sc[2 * kt + 1][0], sl2, -m_use));
-        const float p11 = ex2(fmaf(sc[2 * kt + 1][1], sl2, -m_use));
-        psum += (p00 + p01) + (p10 + p11);
-        pa[kt][0] = pack_bf16(p00, p01);
-        pa[kt][1] = pack_bf16(p10, p11);
+      for (int mt = 0; mt < MT; ++mt) {
+        mx0 = fmaxf(mx0, fmaxf(sT[mt][0], sT[mt][2]));
+        mx1 = fmaxf(mx1, fmaxf(sT[mt][1], sT[mt][3]));
       }
-      l_run = l_run * corr + psum;
-      m_run = m_new;
-      if (__any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
-        for (int i2 = 0; i2 < D / 8; ++i2) { o[i2][0] *= corr; o[i2][1] *= corr; }
+      for (int o = 4; o < 32; o <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
       }
-      // ---- O += P V -------------------------------------------------------------------------------------------
+      const float m_new0 = fmaxf(m_run0, mx0 * sl2), m_new1 = fmaxf(m_run1, mx1 * sl2);
+      const float m_use0 = (m_new0 == -INFINITY) ? 0.f : m_new0;     // all-masked: keep exp2 arguments finite
+      const float m_use1 = (m_new1 == -INFINITY) ? 0.f : m_new1;
+      const float corr0 = ex2(m_run0 - m_use0), corr1 = ex2(m_run1 - m_use1);
+      float psum0 = 0.f, psum1 = 0.f;
+      uint32_t pb[MT][2];                                    // P^T as B fragments: [tokens 2qc.., +8][head qr]
 #pragma unroll
-      for (int kt = 0; kt < KT16; ++kt) {
+      for (int mt = 0; mt < MT; ++mt) {
+        const float p00 = ex2(fmaf(sT[mt][0], sl2, -m_use0));      // token qr,     head 2qc
+        const float p01 = ex2(fmaf(sT[mt][1], sl2, -m_use1));      // token qr,     head 2qc + 1
+        const float p10 = ex2(fmaf(sT[mt][2], sl2, -m_use0));      // token qr + 8, head 2qc
+        const float p11 = ex2(fmaf(sT[mt][3], sl2, -m_use1));
+        psum0 += p00 + p10;
+        psum1 += p01 + p11;
+        pb[mt][0] = movm_t(pack_bf16(p00, p01));             // 8 x 8 transpose across the warp
+        pb[mt][1] = movm_t(pack_bf16(p10, p11));
+      }
+      l_run0 = l_run0 * corr0 + psum0;
+      l_run1 = l_run1 * corr1 + psum1;
+      m_run0 = m_new0;
+      m_run1 = m_new1;
+      if (__any_sync(0xffffffffu, corr0 != 1.f || corr1 != 1.f)) {
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt) { oT[dt][0] *= corr0; oT[dt][1] *= corr1; oT[dt][2] *= corr0; oT[dt][3] *= corr1; }
+      }
+      // ---- O^T += V^T P^T: A = a 16-dim x 16-token block of V^T (ldmatrix.trans), B = P^T ------------------------
+#pragma unroll
+      for (int kt = 0; kt < MT; ++kt) {
         const int row = 16 * kt + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-        for (int dp = 0; dp < D / 16; ++dp) {
-          const int cidx = 2 * dp + (lane >> 4);
+        for (int dt = 0; dt < DT; ++dt) {
+          const int cidx = 2 * dt + (lane >> 4);
           const int hf = cidx >> 3, cc = cidx & 7;
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(vb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), b0, b1, b2, b3);
-          mma_top(o[2 * dp][0], o[2 * dp][1], pa[kt][0], pa[kt][1], b0, b1);
-          mma_top(o[2 * dp + 1][0], o[2 * dp + 1][1], pa[kt][0], pa[kt][1], b2, b3);
+          uint32_t r0, r1, r2, r3;           // (tok 0-7, d 0-7), (tok 8-15, d 0-7), (tok 0-7, d 8-15), (tok 8-15, d 8-15)
+          ldsm_x4_t(vb + hf * HALF_BYTES + row * 128 + ((cc ^ (row & 7)) << 4), r0, r1, r2, r3);
+          mma_full(oT[dt], r0, r2, r1, r3, pb[kt][0], pb[kt][1]);
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_empty + 8 * s);
     }
 
-    // ---- merge the warps' partials of this unit ---------------------------------------------------------------
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    {
-      float* acc = mb_acc + (warp * 8 + qr) * SM::ACC_STRIDE + 2 * qc;
+    // ---- the warp's partials of this unit -> shared memory ---------------------------------------------------------
 #pragma unroll
-      for (int i2 = 0; i2 < D / 8; ++i2) *reinterpret_cast<float2*>(acc + 8 * i2) = make_float2(o[i2][0], o[i2][1]);
-      if (qc == 0) { mb_ml[warp * 16 + qr] = m_run; mb_ml[warp * 16 + 8 + qr] = l_run; }
+    for (int o = 4; o < 32; o <<= 1) {
+      l_run0 += __shfl_xor_sync(0xffffffffu, l_run0, o);
+      l_run1 += __shfl_xor_sync(0xffffffffu, l_run1, o);
+    }
+    {
+      float* acc0 = mb_acc + (warp * 8 + 2 * qc) * SM::ACC_STRIDE + qr;      // head 2 qc, dim qr (+ 8, + 16 dt)
+      float* acc1 = acc0 + SM::ACC_STRIDE;                                    // head 2 qc + 1
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        acc0[16 * dt] = oT[dt][0];
+        acc1[16 * dt] = oT[dt][1];
+        acc0[16 * dt + 8] = oT[dt][2];
+        acc1[16 * dt + 8] = oT[dt][3];
+      }
+      if (qr == 0) {
+        mb_ml[warp * 16 + 2 * qc] = m_run0;
+        mb_ml[warp * 16 + 2 * qc + 1] = m_run1;
+        mb_ml[warp * 16 + 8 + 2 * qc] = l_run0;
+        mb_ml[warp * 16 + 8 + 2 * qc + 1] = l_run1;
+      }
     }
     consumer_sync(NCONS);
 
