@@ -647,13 +647,25 @@ bool make_ring_map(CUtensorMap* map, void* base, long long rows, int D, int tile
 constexpr int NW_DEFAULT = PTENC_ATTN_NW;
 template <int D> struct Pick {
   static constexpr int TILE_N = (D == 128) ? PTENC_ATTN_TILE_N_128 : 64;
-  static constexpr int STAGES = (D == 128) ? PTENC_ATTN_STAGES_128 : 12 / NW_DEFAULT * NW_DEFAULT;
+  static constexpr int STAGES = (D == 128) ? PTENC_ATTN_STAGES_128 : 12;
 };
+// Long launches run under the power cap, and there three consumer warps sustain 2-3 % more bandwidth than four
+// (measured medians of 500+ back-to-back launches: 7B shape 6947 vs 6820 GB/s, Llama shape 7156 vs 6926, 4096-token
+// windows 7060 vs 6858); short launches and short windows (few tiles per unit, more merging per byte) are better off
+// with four (3B shape 6318 vs 6470, 512-token windows 6100 vs 6365).  The choice is made per launch from the
+// number of tiles the call can hold.
+constexpr int NW_LONG = 3;
+inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
+  if (NW_DEFAULT != 4) return false;                    // only when the default was not overridden at build time
+  const long long n_t = (cfg.window + tile_n - 1) / tile_n;
+  const long long tiles = (long long)nl * cfg.batch * cfg.n_kv_heads * n_t;
+  return n_t >= 32 && tiles >= 300000;
+}
 
-template <int D>
+template <int D, int NW>
 cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
                      cudaStream_t st) {
-  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+  constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   const size_t smem = SM::TOTAL + 1024;
   k_attn_bf16<D, TN, NW, STAGES><<<c->attn_grid, (NW + 1) * 32, smem, st>>>(
@@ -662,12 +674,18 @@ cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_
   return cudaGetLastError();
 }
 
-template <int D>
-cudaError_t prepare_t() {
-  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+template <int D, int NW>
+cudaError_t prepare_nw() {
+  constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   return cudaFuncSetAttribute(k_attn_bf16<D, TN, NW, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               SM::TOTAL + 1024);
+}
+template <int D>
+cudaError_t prepare_t() {
+  cudaError_t e = prepare_nw<D, NW_DEFAULT>();
+  if (e == cudaSuccess && NW_DEFAULT != NW_LONG) e = prepare_nw<D, NW_LONG>();
+  return e;
 }
 
 }  // namespace
@@ -691,8 +709,12 @@ bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err) {
 
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
                                    float* lse, cudaStream_t st) {
-  if (c->cfg.head_dim == 128) return launch_t<128>(c, l0, nl, q, active, out, lse, st);
-  return launch_t<64>(c, l0, nl, q, active, out, lse, st);
+  const bool d128 = c->cfg.head_dim == 128;
+  const bool lng = use_long_variant(c->cfg, nl, d128 ? Pick<128>::TILE_N : Pick<64>::TILE_N);
+  if (d128) return lng ? launch_t<128, NW_LONG>(c, l0, nl, q, active, out, lse, st)
+                       : launch_t<128, NW_DEFAULT>(c, l0, nl, q, active, out, lse, st);
+  return lng ? launch_t<64, NW_LONG>(c, l0, nl, q, active, out, lse, st)
+             : launch_t<64, NW_DEFAULT>(c, l0, nl, q, active, out, lse, st);
 }
 
 // ================================================================================================================
