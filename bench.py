@@ -33,7 +33,7 @@ METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0030   # (dram read + write) / algorithmic, ncu, see profiles/
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0029   # (dram read + write) / algorithmic, ncu, see profiles/
 
 
 def workload_cfg(name: str) -> dict:

@@ -32,7 +32,10 @@ def needs_build() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+    """Compiles the sources and links libptenc.so.  Extra nvcc flags (e.g. -DPTENC_ATTN_NW=3 to pin a tunable of the
+    attention kernel for profiling) can be given in the environment variable PTENC_NVCC_FLAGS; they force a rebuild."""
+    extra = os.environ.get("PTENC_NVCC_FLAGS", "").split()
+    if not force and not extra and not needs_build():
         return LIB
     objdir = os.path.join(PKG, "_build")
     os.makedirs(objdir, exist_ok=True)
@@ -40,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for s in SOURCES:
         obj = os.path.join(objdir, s.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c",
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c",
                os.path.join(CSRC, s), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
