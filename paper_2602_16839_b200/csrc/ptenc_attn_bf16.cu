@@ -654,7 +654,10 @@ template <int D> struct Pick {
 // windows 7060 vs 6858); short launches and short windows (few tiles per unit, more merging per byte) are better off
 // with four (3B shape 6318 vs 6470, 512-token windows 6100 vs 6365).  The choice is made per launch from the
 // number of tiles the call can hold.
-constexpr int NW_LONG = 3;
+#ifndef PTENC_ATTN_NW_LONG
+#define PTENC_ATTN_NW_LONG 3
+#endif
+constexpr int NW_LONG = PTENC_ATTN_NW_LONG;
 inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
   if (NW_DEFAULT != 4) return false;                    // only when the default was not overridden at build time
   const long long n_t = (cfg.window + tile_n - 1) / tile_n;
