@@ -2,10 +2,10 @@
  * ptenc.h -- C ABI of the Progressive Thought Encoding decode hot path (sm_100a).
  *
  * One decode step under a fixed-size KV cache, per layer and per sequence:
- *   a1  ring-buffer append / evict           (Sec. 3.2 cache policy D; Sec. 3.3 "until the KV
- *                                             cache is full ... earlier tokens evicted"; Sec. 4.1
- *                                             implementation details: a fraction of the tokens is
- *                                             evicted on saturation)
+ *   a1  ring-buffer append / evict           (Sec. 3.2 cache policy D; Sec. 3.3: decoding fills the
+ *                                             cache, then the policy removes the oldest tokens;
+ *                                             Sec. 4.1 implementation details: a fraction of the
+ *                                             tokens leaves at once when the cache saturates)
  *   a2  grouped-query decode attention       (Sec. 3.1, the two attention equations: the new query
  *                                             attends over the cache including the new token)
  *   a3  progressive encode of evicted tokens (Sec. 3.3, Eq. (3): S' = ((W^a_Q q_g)(W^a_K K_e)^T)(W^a_V V_e);
@@ -64,6 +64,9 @@ extern "C" {
 #define PTENC_NORM_FROBENIUS 1    /* whole state divided by max(||S||_F, 1e-12)                       */
 #define PTENC_NORM_NONE      2
 
+#define PTENC_POLICY_FIFO    0    /* sliding window: the oldest tokens leave (Sec. 3.3, the policy of the paper's runs) */
+#define PTENC_POLICY_SCORE   1    /* the tokens that received the least attention so far leave (Sec. 4.3, token dropping) */
+
 typedef struct ptenc_cache ptenc_cache;   /* opaque host handle */
 
 typedef struct {
@@ -80,7 +83,11 @@ typedef struct {
   int32_t normalize_mode;  /* PTENC_NORM_*                                                          */
   int32_t encode_enabled;  /* 0: state stays at its initial value ("Global-Only" ablation, Sec. 4.3) */
   int32_t device;          /* CUDA device ordinal the workspace lives on                            */
-  int32_t reserved[3];     /* must be zero                                                          */
+  int32_t attn_consumer_warps; /* tuning knob of the bf16 tensor-core attention kernel: 0 = chosen per launch
+                                  (three warps on long launches of long windows, four otherwise), 3 or 4 = fixed  */
+  int32_t policy;          /* PTENC_POLICY_*: which tokens leave when the cache is full                       */
+  int32_t recent;          /* PTENC_POLICY_SCORE only: the newest `recent` tokens are never evicted (0..W-1);
+                              must be 0 under PTENC_POLICY_FIFO                                               */
 } ptenc_config;
 
 /* Bytes of device workspace a cache with this configuration needs.  Host only, launches nothing.
@@ -100,7 +107,9 @@ PTENC_API int ptenc_cache_destroy(ptenc_cache* c);
 
 /* Empties the caches of the sequences with seq_mask[b] != 0 (NULL = all) in every layer (ring and pinned prompt
  * entries) and puts their state back to the layer's initial state S_0 (zero when no encoder was set).  With
- * seq_mask == NULL the device status word is cleared too. */
+ * seq_mask == NULL the device status word and the attention kernel's split-unit arrival counters are cleared too,
+ * so a cache whose status word reported a launch that gave up (bounded wait ran out, inconsistent ring state)
+ * is fully usable again after this call. */
 PTENC_API int ptenc_cache_reset(ptenc_cache* c, const uint8_t* seq_mask /*[B], nullable*/, void* stream);
 
 /* Encoder set-up for one layer (Sec. 3.3): stores W^a_K, W^a_V, computes Q_a = q_g W^a_Q^T [G,r] and the
@@ -210,6 +219,30 @@ PTENC_API int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status /*host, out
 PTENC_API int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn /*host, out*/,
                                int32_t* attn_grid /*host, out*/, int32_t* tensor_core_encode /*host, out*/);
 
+/* What the next attention launch through this handle would run for `layer` (-1 = all layers in one call), host only,
+ * every output nullable: *consumer_warps = warps that consume K/V tiles in the tensor-core kernel (3 or 4; chosen
+ * per launch from the tiles the call can hold unless ptenc_config.attn_consumer_warps fixes it), *tile_tokens =
+ * tokens per K/V tile, *stages = shared-memory pipeline stages.  All three are 0 when the shape-generic kernel
+ * serves the cache. */
+PTENC_API int ptenc_attn_launch_info(ptenc_cache* c, int layer, int32_t* consumer_warps /*host, out*/,
+                                     int32_t* tile_tokens /*host, out*/, int32_t* stages /*host, out*/);
+
+/* Where one part of the decode state lives inside the workspace (host only): byte offset from the workspace base
+ * and size.  The whole workspace is the checkpoint; this map lets a tool save, inspect or patch one part of it.
+ * PTENC_EINVAL for an unknown region. */
+#define PTENC_REGION_K        0   /* key rings   [L][B][H_kv][W][D], storage dtype                           */
+#define PTENC_REGION_V        1   /* value rings                                                             */
+#define PTENC_REGION_HEAD     2   /* int32 [L][B]                                                            */
+#define PTENC_REGION_COUNT    3   /* int32 [L][B]                                                            */
+#define PTENC_REGION_NAPP     4   /* int64 [L][B]                                                            */
+#define PTENC_REGION_NPINNED  5   /* int32 [L][B]                                                            */
+#define PTENC_REGION_STATE    6   /* fp32  [L][B][G][r]                                                      */
+#define PTENC_REGION_TICKETS  7   /* int32 [L][B][H_kv]: split-unit arrival counters of the attention kernel, zero
+                                     between launches                                                        */
+#define PTENC_REGION_STATUS   8   /* int32: the device status word                                           */
+PTENC_API int ptenc_workspace_region(ptenc_cache* c, int region, size_t* offset /*host, out*/,
+                                     size_t* bytes /*host, out*/);
+
 /* Timing hook.  The next attention launch made through this handle (by ptenc_decode_attn, ptenc_decode_step
  * or ptenc_decode_step_host) records the two cudaEvent_t (passed as void*) on its stream immediately
  * before and after the attention kernel; the hook is then cleared.  NULL, NULL cancels it. */
@@ -228,17 +261,22 @@ PTENC_API int ptenc_launch_count(ptenc_cache* c, int64_t* n_launches /*host, out
  * The kernel's scratch (split-K partials, arrival tickets, a status word) lives in a 2,392,320-byte device array
  * that is part of the library image: every GPU that loads the library holds it until the process exits.
  *
- * Computes exactly what ptenc_decode_attn computes with layer = -1, with the same kernel.
- *   cfg      host; n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, dtype, device are read.  Only the
- *            tensor-core kernel has this variant: dtype bf16, head_dim 64 or 128, n_q_heads/n_kv_heads <= 8,
- *            else PTENC_ESHAPE.
+ * Computes exactly what ptenc_decode_attn computes with layer = -1, with the same kernel and the same choice of
+ * instantiation (consumer warps per launch, see ptenc_attn_launch_info).
+ *   cfg      host; n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, dtype, device, attn_consumer_warps are
+ *            read.  Only the tensor-core kernel has this variant: dtype bf16, head_dim 64 or 128,
+ *            n_q_heads/n_kv_heads <= 8, else PTENC_ESHAPE.  cfg->device must be the calling thread's current device
+ *            (PTENC_EINVAL otherwise): the entry does not switch devices.
  *   K, V     device, [L][B][H_kv][W][D] bf16, 16-byte aligned: the rings.  Slots that hold no live token must
  *            contain finite values (e.g. zeros).
  *   head, count  device int32 [L][B]: slot of the oldest live token and number of live tokens of each ring;
  *            live slots are head, head+1, ... (mod W).
  *   q, out   device, [L][B][H_q][D] bf16; active [B] bytes or NULL; lse_out [L][B][H_q] fp32 or NULL.
  *   status_out  device int32 or NULL: receives the kernel's status word (0 = clean) once the call has run.
- * Limits: n_layers * batch * n_kv_heads <= 65536, else PTENC_ELIMIT (nothing is launched).
+ *            A ring whose head or count is out of range (head outside [0, W), count outside [0, W]) is skipped:
+ *            its output rows are not written and the status word gets bit 2.
+ * Limits: n_layers * batch * n_kv_heads <= 65536 units and n_layers * batch * n_kv_heads * window < 2^31 rows, else
+ * PTENC_ELIMIT (nothing is launched).
  * The first call on a device resolves the array's device address and sets kernel attributes (once per device,
  * with that device current); make that first call before any stream capture.  Every call on a device shares the
  * one array, and the array keeps the previous call's contents: the entry clears the status word and the tickets on

@@ -19,17 +19,22 @@ PTENC_OK, PTENC_EINVAL, PTENC_ESHAPE, PTENC_EALIGN, PTENC_EWORKSPACE, PTENC_ECUD
 PTENC_ELIMIT = -7
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 NORM_ROW_L2, NORM_FROBENIUS, NORM_NONE = 0, 1, 2
+POLICY_FIFO, POLICY_SCORE = 0, 1
+(REGION_K, REGION_V, REGION_HEAD, REGION_COUNT, REGION_NAPP, REGION_NPINNED, REGION_STATE, REGION_TICKETS,
+ REGION_STATUS) = range(9)
 
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
            "ptenc_set_encoder", "ptenc_prefill", "ptenc_get_pinned", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_lora_apply", "ptenc_decode_step",
            "ptenc_host_staging_bytes", "ptenc_decode_step_host",
-           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count", "ptenc_strerror"]
+           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_attn_launch_info",
+           "ptenc_workspace_region", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count",
+           "ptenc_strerror"]
 
 
 class PtencConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "window", "evict_chunk", "n_global",
-        "rank", "dtype", "normalize_mode", "encode_enabled", "device")] + [("reserved", ctypes.c_int32 * 3)]
+        "rank", "dtype", "normalize_mode", "encode_enabled", "device", "attn_consumer_warps", "policy", "recent")]
 
 
 class PtencError(RuntimeError):
@@ -64,6 +69,8 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_get_state.argtypes = [vp, i32, vp, vp]
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_cache_info.argtypes = [vp] + [ctypes.POINTER(ctypes.c_int32)] * 3
+    lib.ptenc_attn_launch_info.argtypes = [vp, i32] + [ctypes.POINTER(ctypes.c_int32)] * 3
+    lib.ptenc_workspace_region.argtypes = [vp, i32, ctypes.POINTER(u64), ctypes.POINTER(u64)]
     lib.ptenc_time_next_attn.argtypes = [vp, vp, vp]
     lib.ptenc_attn_rings_static.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ptenc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
@@ -98,12 +105,14 @@ def _stream() -> int:
 
 
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, evict_chunk=1, n_global=32,
-                rank=32, dtype="bf16", normalize_mode=0, encode_enabled=1, device=0) -> PtencConfig:
+                rank=32, dtype="bf16", normalize_mode=0, encode_enabled=1, device=0, attn_consumer_warps=0,
+                policy=POLICY_FIFO, recent=0) -> PtencConfig:
     c = PtencConfig()
     c.n_layers, c.batch, c.n_q_heads, c.n_kv_heads, c.head_dim = n_layers, batch, n_q_heads, n_kv_heads, head_dim
     c.window, c.evict_chunk, c.n_global, c.rank = window, evict_chunk, n_global, rank
     c.dtype = {"fp32": DTYPE_FP32, "bf16": DTYPE_BF16}[dtype] if isinstance(dtype, str) else int(dtype)
     c.normalize_mode, c.encode_enabled, c.device = normalize_mode, encode_enabled, device
+    c.attn_consumer_warps, c.policy, c.recent = attn_consumer_warps, policy, recent
     return c
 
 
@@ -226,6 +235,19 @@ class Cache:
         a, b, e = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
         _check(lib.ptenc_cache_info(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(e)), "ptenc_cache_info")
         return {"tensor_core_attn": bool(a.value), "attn_grid": int(b.value), "tensor_core_encode": bool(e.value)}
+
+    def attn_launch_info(self, layer=-1) -> dict:
+        w, t, s = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(lib.ptenc_attn_launch_info(self._h, layer, ctypes.byref(w), ctypes.byref(t), ctypes.byref(s)),
+               "ptenc_attn_launch_info")
+        return {"consumer_warps": int(w.value), "tile_tokens": int(t.value), "stages": int(s.value)}
+
+    def workspace_region(self, region: int):
+        """(device pointer, bytes) of one part of the decode state inside the workspace."""
+        off, n = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        _check(lib.ptenc_workspace_region(self._h, int(region), ctypes.byref(off), ctypes.byref(n)),
+               "ptenc_workspace_region")
+        return self._ws_ptr + int(off.value), int(n.value)
 
     def time_next_attn(self, ev_begin, ev_end):
         """ev_begin/ev_end: torch.cuda.Event(enable_timing=True) that have been recorded once (so that their

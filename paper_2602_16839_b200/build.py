@@ -23,19 +23,33 @@ def _nvcc() -> str:
     return exe
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+STAMP = os.path.join(PKG, "libptenc.flags")     # travels with the library, unlike the object folder
+
+
+def _stamp(extra) -> str:
+    return " ".join([*NVCC_FLAGS, *extra])
+
+
+def needs_build(extra=()) -> bool:
+    """True when the library is missing, older than a source, or was built with other flags than asked for now
+    (so a library built with extra tunables is never mistaken for the default one)."""
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
+    with open(STAMP) as f:
+        if f.read().strip() != _stamp(extra):
+            return True
     t = os.path.getmtime(LIB)
     deps = [os.path.join(CSRC, s) for s in SOURCES] + HEADERS
     return any(os.path.getmtime(d) > t for d in deps)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compiles the sources and links libptenc.so.  Extra nvcc flags (e.g. -DPTENC_ATTN_NW=3 to pin a tunable of the
-    attention kernel for profiling) can be given in the environment variable PTENC_NVCC_FLAGS; they force a rebuild."""
+    """Compiles the sources and links libptenc.so.  Extra nvcc flags (e.g. -DPTENC_ATTN_STAGES_128=8 to pin a tunable
+    of the attention kernel for profiling) can be given in the environment variable PTENC_NVCC_FLAGS.  The flags of
+    the last build are recorded beside the library; a build with other flags, or the default build after a flagged
+    one, recompiles."""
     extra = os.environ.get("PTENC_NVCC_FLAGS", "").split()
-    if not force and not extra and not needs_build():
+    if not force and not needs_build(extra):
         return LIB
     objdir = os.path.join(PKG, "_build")
     os.makedirs(objdir, exist_ok=True)
@@ -61,6 +75,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}")
+    with open(STAMP, "w") as f:
+        f.write(_stamp(extra) + "\n")
     return LIB
 
 

@@ -28,7 +28,9 @@ int validate_config(const ptenc_config* c) {
   if (c->normalize_mode < 0 || c->normalize_mode > 2) return PTENC_EINVAL;
   if (c->encode_enabled != 0 && c->encode_enabled != 1) return PTENC_EINVAL;
   if (c->device < 0) return PTENC_EINVAL;
-  if (c->reserved[0] != 0 || c->reserved[1] != 0 || c->reserved[2] != 0) return PTENC_EINVAL;
+  if (c->attn_consumer_warps != 0 && c->attn_consumer_warps != 3 && c->attn_consumer_warps != 4) return PTENC_EINVAL;
+  if (c->policy != PTENC_POLICY_FIFO) return PTENC_EINVAL;
+  if (c->recent != 0) return PTENC_EINVAL;
   if (c->n_q_heads % c->n_kv_heads != 0) return PTENC_ESHAPE;
   if (c->head_dim % 8 != 0 || c->head_dim > 256) return PTENC_ESHAPE;
   if (c->n_global < 1 || c->n_global > 128 || c->rank < 1 || c->rank > 128) return PTENC_ESHAPE;
@@ -215,7 +217,14 @@ int ptenc_cache_destroy(ptenc_cache* c) {
 
 int ptenc_cache_reset(ptenc_cache* c, const uint8_t* seq_mask, void* stream) {
   if (c == nullptr) return PTENC_EINVAL;
-  return ptenc_launch_reset(c, seq_mask, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (seq_mask == nullptr) {
+    // A launch that gave up part-way (a bounded wait ran out, the schedule did not add up) can leave arrival counts
+    // of split units behind; the full reset is the documented way back, so it clears them with the status word.
+    const PtencDev& d = c->dev;
+    if (cudaMemsetAsync(d.tickets, 0, (size_t)d.L * d.B * d.Hkv * 4, st) != cudaSuccess) return PTENC_ECUDA;
+  }
+  return ptenc_launch_reset(c, seq_mask, st) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_set_encoder(ptenc_cache* c, int layer, const void* Wq_a, const void* Wk_a, const void* Wv_a,
@@ -495,6 +504,39 @@ int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn, int32_t* attn_gr
   if (tensor_core_attn) *tensor_core_attn = c->fast_attn ? 1 : 0;
   if (attn_grid) *attn_grid = c->fast_attn ? c->attn_grid : 0;
   if (tensor_core_encode) *tensor_core_encode = c->tc_encode ? 1 : 0;
+  return PTENC_OK;
+}
+
+int ptenc_attn_launch_info(ptenc_cache* c, int layer, int32_t* consumer_warps, int32_t* tile_tokens,
+                           int32_t* stages) {
+  int l0, nl;
+  int rc = check_layer(c, layer, &l0, &nl);
+  if (rc != PTENC_OK) return rc;
+  int nw = 0, tn = 0, ns = 0;
+  if (c->fast_attn) ptenc_attn_bf16_plan(c, nl, &nw, &tn, &ns);
+  if (consumer_warps) *consumer_warps = nw;
+  if (tile_tokens) *tile_tokens = tn;
+  if (stages) *stages = ns;
+  return PTENC_OK;
+}
+
+int ptenc_workspace_region(ptenc_cache* c, int region, size_t* offset, size_t* bytes) {
+  if (c == nullptr || offset == nullptr || bytes == nullptr) return PTENC_EINVAL;
+  const Layout lay = make_layout(&c->cfg);
+  const size_t elt = c->dev.elt, L = c->dev.L, B = c->dev.B;
+  const size_t ring = L * B * (size_t)c->dev.Hkv * c->dev.W * c->dev.D * elt;
+  switch (region) {
+    case PTENC_REGION_K: *offset = lay.K; *bytes = ring; break;
+    case PTENC_REGION_V: *offset = lay.V; *bytes = ring; break;
+    case PTENC_REGION_HEAD: *offset = lay.head; *bytes = L * B * 4; break;
+    case PTENC_REGION_COUNT: *offset = lay.count; *bytes = L * B * 4; break;
+    case PTENC_REGION_NAPP: *offset = lay.n_app; *bytes = L * B * 8; break;
+    case PTENC_REGION_NPINNED: *offset = lay.n_sink; *bytes = L * B * 4; break;
+    case PTENC_REGION_STATE: *offset = lay.S; *bytes = L * B * (size_t)c->dev.G * c->dev.r * 4; break;
+    case PTENC_REGION_TICKETS: *offset = lay.tickets; *bytes = L * B * (size_t)c->dev.Hkv * 4; break;
+    case PTENC_REGION_STATUS: *offset = lay.status; *bytes = 4; break;
+    default: return PTENC_EINVAL;
+  }
   return PTENC_OK;
 }
 

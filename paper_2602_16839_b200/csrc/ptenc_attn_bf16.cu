@@ -5,12 +5,12 @@
 // is read once per step and there is no reuse between steps.
 //
 // Design
-//  * Persistent grid, one CTA per SM.  The work is the flat list of 64-token tiles of every
-//    (layer, sequence, KV head) unit that has live tokens; CTA c takes the contiguous share
+//  * Persistent grid, one CTA per SM.  The work is the flat list of K/V tiles (32 tokens at head_dim 128, 64 at
+//    head_dim 64) of every (layer, sequence, KV head) unit that has live tokens; CTA c takes the contiguous share
 //    [c*T/n, (c+1)*T/n) of the T tiles, so no SM idles in a tail wave whatever B*H_kv is (split-K at tile
 //    granularity, sized to the machine).
-//  * A producer warp streams K and V tiles with TMA (cp.async.bulk.tensor, 128-byte swizzle, no
-//    multicast) into a ring of shared-memory stages guarded by full/empty mbarriers.
+//  * A producer warp streams K and V tiles with TMA (cp.async.bulk.tensor, 128-byte swizzle; plain per-CTA loads
+//    of this GPU's own memory) into a ring of shared-memory stages guarded by full/empty mbarriers.
 //  * Each consumer warp owns whole tiles (tile n of the CTA goes to warp n mod NW, stage n mod STAGES; STAGES
 //    is a multiple of NW so a stage always has the same consumer warp and its full/empty barriers advance
 //    one phase per visit -- a warp can never be a phase ahead of a barrier it polls).  The two products run on
@@ -216,6 +216,9 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     en.sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;
     const int cap = W - en.sink;
     if (en.sink < 0 || cap < 1 || en.head < 0 || en.head >= cap || en.count < 0 || en.count > cap) {
+      // a ring state outside its range (corrupt workspace, or bad head/count arrays handed to the static-scratch
+      // entry): the sequence is skipped, nothing of it is loaded, and the status word says so
+      atomicOr(p.status, PTENC_ST_BAD_INDEX);
       en.head = en.count = en.sink = 0;
       return en;
     }
@@ -657,12 +660,21 @@ template <int D> struct Pick {
 #ifndef PTENC_ATTN_NW_LONG
 #define PTENC_ATTN_NW_LONG 3
 #endif
+#ifndef PTENC_ATTN_LONG_MIN_TILES_PER_UNIT
+#define PTENC_ATTN_LONG_MIN_TILES_PER_UNIT 32
+#endif
+#ifndef PTENC_ATTN_LONG_MIN_TILES
+#define PTENC_ATTN_LONG_MIN_TILES 300000
+#endif
 constexpr int NW_LONG = PTENC_ATTN_NW_LONG;
 inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
+  // ptenc_config.attn_consumer_warps fixes the choice when it names one of the two instantiations
+  if (cfg.attn_consumer_warps == NW_LONG) return true;
+  if (cfg.attn_consumer_warps == NW_DEFAULT) return false;
   if (NW_DEFAULT != 4) return false;                    // only when the default was not overridden at build time
   const long long n_t = (cfg.window + tile_n - 1) / tile_n;
   const long long tiles = (long long)nl * cfg.batch * cfg.n_kv_heads * n_t;
-  return n_t >= 32 && tiles >= 300000;
+  return n_t >= PTENC_ATTN_LONG_MIN_TILES_PER_UNIT && tiles >= PTENC_ATTN_LONG_MIN_TILES;
 }
 
 template <int D, int NW>
@@ -708,6 +720,14 @@ bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err) {
   c->attn_grid = c->sm_count * PTENC_ATTN_CTAS_PER_SM;
   if (2 * c->attn_grid > c->dev.part_slots) c->attn_grid = c->dev.part_slots / 2;
   return true;
+}
+
+void ptenc_attn_bf16_plan(const ptenc_cache* c, int nl, int* consumer_warps, int* tile_tokens, int* stages) {
+  const bool d128 = c->cfg.head_dim == 128;
+  const int tn = d128 ? Pick<128>::TILE_N : Pick<64>::TILE_N;
+  *consumer_warps = use_long_variant(c->cfg, nl, tn) ? NW_LONG : NW_DEFAULT;
+  *tile_tokens = tn;
+  *stages = d128 ? Pick<128>::STAGES : Pick<64>::STAGES;
 }
 
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
@@ -777,10 +797,10 @@ cudaError_t static_setup(int device, StaticDevice** out) {
   return cudaSuccess;
 }
 
-template <int D>
+template <int D, int NW>
 cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const CUtensorMap& tmV, int grid, int nl,
                             const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
-  constexpr int NW = NW_DEFAULT, STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
+  constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   k_attn_bf16<D, TN, NW, STAGES><<<grid, (NW + 1) * 32, SM::TOTAL + 1024, st>>>(
       dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
@@ -798,6 +818,8 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   if (cfg->n_layers <= 0 || cfg->batch <= 0 || cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->window <= 0 ||
       cfg->device < 0)
     return PTENC_EINVAL;
+  if (cfg->attn_consumer_warps != 0 && cfg->attn_consumer_warps != 3 && cfg->attn_consumer_warps != 4)
+    return PTENC_EINVAL;
   if (cfg->n_q_heads % cfg->n_kv_heads != 0) return PTENC_ESHAPE;
   if (cfg->dtype != PTENC_DTYPE_BF16 || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
       cfg->n_q_heads / cfg->n_kv_heads > 8)
@@ -809,7 +831,10 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
         reinterpret_cast<uintptr_t>(out)) & 15) != 0)
     return PTENC_EALIGN;
 
-  if (cudaSetDevice(cfg->device) != cudaSuccess) return PTENC_ECUDA;
+  // Like every other entry point this one leaves the caller's current device alone: cfg->device has to be current.
+  int cur_dev = -1;
+  if (cudaGetDevice(&cur_dev) != cudaSuccess) return PTENC_ECUDA;
+  if (cur_dev != cfg->device) return PTENC_EINVAL;
   StaticDevice* sd = nullptr;
   if (static_setup(cfg->device, &sd) != cudaSuccess) return PTENC_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -838,9 +863,15 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
 
   // The array keeps whatever the last call left: the status word and the tickets must start at zero.
   if (cudaMemsetAsync(sd->scratch, 0, STATIC_OFF_TICKETS + (size_t)units * 4, st) != cudaSuccess) return PTENC_ECUDA;
-  cudaError_t e = cfg->head_dim == 128
-                      ? launch_static_t<128>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
-                      : launch_static_t<64>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
+  // the same choice of instantiation as ptenc_decode_attn makes for a call over all layers
+  const bool lng = use_long_variant(*cfg, cfg->n_layers, tile_n);
+  cudaError_t e;
+  if (cfg->head_dim == 128)
+    e = lng ? launch_static_t<128, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
+            : launch_static_t<128, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
+  else
+    e = lng ? launch_static_t<64, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
+            : launch_static_t<64, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
   if (e != cudaSuccess) return PTENC_ECUDA;
   if (status_out != nullptr &&
       cudaMemcpyAsync(status_out, d.status, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)

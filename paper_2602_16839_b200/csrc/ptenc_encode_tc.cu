@@ -9,7 +9,7 @@
 // CTAs (two per SM) walk the (layer, sequence) units that have evicted rows; per CTA:
 //  * warp 0 (one lane): TMA producer.  Per pipeline item it loads a [rows x 64] slab of the evicted K (or V) rows
 //    and the matching [r x 64] slab of W^a_K (or W^a_V), both K-major with the 128-byte swizzle, into a stage
-//    guarded by full/empty mbarriers.  Plain loads, no multicast.
+//    guarded by full/empty mbarriers.  Plain per-CTA loads of this GPU's own memory.
 //  * warp 1 (one lane): issues tcgen05.mma (M = 128 token rows, N = r, K = 16, bf16 x bf16 -> fp32) with the
 //    accumulators in tensor memory: K_a in columns [0, r), V_a in [r, 2r) of one of two buffers, so the epilogue
 //    of a 128-token tile overlaps the loads and MMAs of the next one.  tcgen05.commit releases the stages and

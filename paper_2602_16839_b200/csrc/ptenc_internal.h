@@ -99,6 +99,8 @@ cudaError_t ptenc_launch_encode_tc(ptenc_cache* c, int l0, int nl, const void* K
 // Host-side preparation of the fast attention path (tensor maps, attributes).  Returns false when the
 // shape is not covered, in which case the generic kernel serves it.
 bool ptenc_attn_bf16_prepare(ptenc_cache* c, cudaError_t* err);
+// The instantiation a launch over `nl` layers would use: consumer warps, tokens per tile, pipeline stages.
+void ptenc_attn_bf16_plan(const ptenc_cache* c, int nl, int* consumer_warps, int* tile_tokens, int* stages);
 
 // Kernel attributes are per device: a launcher sets them the first time it runs on a device.
 constexpr int PTENC_MAX_DEVICES = 64;

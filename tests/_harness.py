@@ -21,7 +21,7 @@ class Pair:
 
     def __init__(self, pt, *, n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, evict_chunk=1,
                  n_global=8, rank=8, dtype="bf16", normalize_mode=0, encode_enabled=1, seed=0,
-                 kv_scale=1.0, set_encoder=True, global_kv=True):
+                 kv_scale=1.0, set_encoder=True, global_kv=True, attn_consumer_warps=0):
         self.pt = pt
         self.shape = dict(n_layers=n_layers, batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads,
                           head_dim=head_dim)
@@ -30,8 +30,11 @@ class Pair:
         self.gen = SynthInputs(seed=seed, dtype=dtype, n_global=n_global, rank=rank, kv_scale=kv_scale,
                                device="cuda:0", **self.shape)
         cfg = pt.make_config(window=window, evict_chunk=evict_chunk, n_global=n_global, rank=rank, dtype=dtype,
-                             normalize_mode=normalize_mode, encode_enabled=encode_enabled, **self.shape)
+                             normalize_mode=normalize_mode, encode_enabled=encode_enabled,
+                             attn_consumer_warps=attn_consumer_warps, **self.shape)
         self.cache = pt.Cache(cfg)
+        if attn_consumer_warps and self.cache.info()["tensor_core_attn"]:
+            assert self.cache.attn_launch_info(-1)["consumer_warps"] == attn_consumer_warps
         self.orc = OracleCache(window=window, evict_chunk=evict_chunk, n_global=n_global, rank=rank,
                                normalize_mode=normalize_mode, encode_enabled=encode_enabled, **self.shape)
         if set_encoder:
@@ -42,6 +45,8 @@ class Pair:
                 self.cache.set_encoder(l, P["Wq_a"], P["Wk_a"], P["Wv_a"], P["q_g"], P["k_g"], P["v_g"])
                 self.orc.set_encoder(l, **{k: (None if v is None else np64(v)) for k, v in P.items()})
         self.out = torch.zeros(n_layers, batch, n_q_heads, head_dim, dtype=self.cache.torch_dtype, device="cuda:0")
+        self.out2 = torch.zeros_like(self.out)
+        self.lse = torch.zeros(n_layers, batch, n_q_heads, dtype=torch.float32, device="cuda:0")
 
     def close(self):
         self.cache.close()
@@ -97,15 +102,29 @@ class Pair:
                 self.cache.append_evict(layer, k[sl], v[sl], act_dev)
                 self.cache.encode(layer)
                 self.cache.decode_attn(layer, q[sl], self.out[sl], act_dev)
-        worst = 0.0
+        if check:
+            # the attention alone once more on the same cache (it changes nothing): same outputs, plus the fp32
+            # log-sum-exp, which is far more sensitive to a mis-counted tile than the rounded outputs are
+            self.out2.zero_()
+            self.lse.zero_()
+            for layer in layers:
+                sl = slice(None) if layer == -1 else layer
+                self.cache.decode_attn(layer, q[sl], self.out2[sl], act_dev, self.lse[sl])
+        worst = worst_lse = 0.0
         qn, kn, vn = np64(q), np64(k), np64(v)
         outn = np64(self.out)
+        lsen = np64(self.lse)
         for l in range(self.L):
             o_ref, lse_ref, rec = self.orc.decode_step(l, qn[l], kn[l], vn[l], active)
             if check:
                 m = np.ones(self.B, bool) if active is None else np.asarray(active, bool)
+                m = m & ((self.orc.ring(l)[1] + self.orc.pinned_count(l)) > 0)
                 if m.any():
                     worst = max(worst, np.abs(outn[l][m] - o_ref[m]).max())
+                    worst_lse = max(worst_lse, np.abs(lsen[l][m] - lse_ref[m]).max())
         if check:
             assert worst <= TOL_OUT[self.dtype], (t, worst)
+            assert worst_lse <= TOL_LSE[self.dtype], (t, worst_lse)
+            ma = slice(None) if active is None else torch.as_tensor(np.asarray(active, bool), device="cuda:0")
+            assert torch.equal(self.out[:, ma], self.out2[:, ma]), t
         return worst

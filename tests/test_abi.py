@@ -74,8 +74,10 @@ def test_create_rejects_null_misaligned_and_small_workspace():
     assert pt.lib.ptenc_cache_create(ctypes.byref(cfg), None, 1 << 30, None, ctypes.byref(h)) == pt.binding.PTENC_EINVAL
     assert pt.lib.ptenc_cache_create(ctypes.byref(cfg), 1024 + 16, 1 << 30, None, ctypes.byref(h)) == pt.binding.PTENC_EALIGN
     assert pt.lib.ptenc_cache_create(ctypes.byref(cfg), 4096, 1000, None, ctypes.byref(h)) == pt.binding.PTENC_EWORKSPACE
-    cfg.reserved[1] = 5
-    assert pt.lib.ptenc_cache_create(ctypes.byref(cfg), 4096, 1 << 30, None, ctypes.byref(h)) == pt.binding.PTENC_EINVAL
+    for field, bad in (("attn_consumer_warps", 5), ("policy", 9), ("recent", -1)):
+        cfg = pt.make_config(**GOOD)
+        setattr(cfg, field, bad)
+        assert pt.lib.ptenc_cache_create(ctypes.byref(cfg), 4096, 1 << 30, None, ctypes.byref(h)) == pt.binding.PTENC_EINVAL
 
 
 def test_null_handle_is_an_error_not_a_crash():

@@ -49,13 +49,18 @@ def test_tiny_fp32_exhaustive():
     p.close()
 
 
-@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+# storage dtype and, for bf16, the consumer-warp count of the tensor-core attention kernel: 0 = the library's choice
+# (four at these sizes), 3 = the instantiation that long launches of long windows use
+KERNELS = [("fp32", 0), ("bf16", 0), ("bf16", 3)]
+
+
+@pytest.mark.parametrize("dtype,warps", KERNELS)
 @pytest.mark.parametrize("Hq,Hkv", [(1, 1), (4, 1), (7, 1), (8, 2), (14, 2), (12, 3)])
-def test_small_shapes_ragged(dtype, Hq, Hkv):
+def test_small_shapes_ragged(dtype, warps, Hq, Hkv):
     """Query-group sizes 1,4,7,8; window not a power of two; sequences active at random."""
     rng = np.random.default_rng(Hq * 10 + Hkv)
     p = Pair(pt, n_layers=2, batch=5, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=64 if dtype == "fp32" else 128,
-             window=37, evict_chunk=1, dtype=dtype, seed=3)
+             window=37, evict_chunk=1, dtype=dtype, seed=3, attn_consumer_warps=warps)
     for t in range(37 * 2 + 11):
         active = (rng.random(5) < 0.8).astype(np.uint8)
         if t == 0:
@@ -69,12 +74,12 @@ def test_small_shapes_ragged(dtype, Hq, Hkv):
     p.close()
 
 
-@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("dtype,warps", KERNELS)
 @pytest.mark.parametrize("W,E", [(1, 1), (2, 1), (3, 2), (5, 5), (64, 16), (100, 25), (100, 100), (130, 1), (257, 65)])
-def test_windows_and_chunks(dtype, W, E):
+def test_windows_and_chunks(dtype, warps, W, E):
     """E in {1, ceil(W/4), W}; W = 1 returns v of the newest token; ragged tile tails."""
     p = Pair(pt, n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 32,
-             window=W, evict_chunk=E, dtype=dtype, seed=W)
+             window=W, evict_chunk=E, dtype=dtype, seed=W, attn_consumer_warps=warps)
     T = min(3 * W + 5, 2 * W + 70)
     for t in range(T):
         p.step(t)
@@ -110,10 +115,11 @@ def test_fused_step_equals_three_calls(dtype, E, batch):
         x.close()
 
 
-def test_bf16_multi_tile_lse():
-    """Several 64-token tiles plus a tail, all query heads of a 7-group, lse output."""
+@pytest.mark.parametrize("warps", [0, 3])
+def test_bf16_multi_tile_lse(warps):
+    """Several 32-token tiles plus a tail, all query heads of a 7-group, lse output."""
     p = Pair(pt, n_layers=2, batch=3, n_q_heads=28, n_kv_heads=4, head_dim=128, window=333, dtype="bf16", seed=11,
-             n_global=32, rank=32)
+             n_global=32, rank=32, attn_consumer_warps=warps)
     lse = torch.empty(2, 3, 28, dtype=torch.float32, device="cuda")
     for t in range(333 + 80):
         p.step(t)
@@ -229,9 +235,11 @@ def test_tensor_core_kernel_serves_bf16_shapes():
     cache.close()
 
 
-def test_split_units_many_tiles_per_cta():
+@pytest.mark.parametrize("warps", [0, 3])
+def test_split_units_many_tiles_per_cta(warps):
     """Enough tiles that every CTA streams many pipeline rounds and most units are split between CTAs."""
-    p = Pair(pt, n_layers=2, batch=7, n_q_heads=28, n_kv_heads=4, head_dim=128, window=1500, dtype="bf16", seed=21)
+    p = Pair(pt, n_layers=2, batch=7, n_q_heads=28, n_kv_heads=4, head_dim=128, window=1500, dtype="bf16", seed=21,
+             attn_consumer_warps=warps)
     # fill quickly: same synthetic stream on both sides, outputs checked at chosen steps only
     for t in range(1500 + 30):
         chk = t in (0, 1, 63, 64, 65, 700, 1499, 1500, 1501, 1529)
@@ -331,14 +339,14 @@ def test_host_buffer_step_equals_device_step(dtype, L):
     a.close(); b.close()
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("dtype,warps", KERNELS)
 @pytest.mark.parametrize("W,E,prompts", [(37, 1, [0, 1, 17, 36, 5]), (96, 24, [0, 33, 64, 95, 80]),
                                          (200, 50, [130, 7, 0, 199, 64])])
-def test_pinned_prompt_and_sliding_window_over_the_rest(dtype, W, E, prompts):
+def test_pinned_prompt_and_sliding_window_over_the_rest(dtype, warps, W, E, prompts):
     """Prompt lengths from none to W - 1 (a single sliding slot), chunks larger than the remaining capacity, tiles
     that straddle the end of the pinned part: outputs, eviction reports, ring and state against the oracle."""
     p = Pair(pt, n_layers=2, batch=5, n_q_heads=8, n_kv_heads=2, head_dim=128 if dtype == "bf16" else 64,
-             window=W, evict_chunk=E, dtype=dtype, seed=W, n_global=16, rank=16)
+             window=W, evict_chunk=E, dtype=dtype, seed=W, n_global=16, rank=16, attn_consumer_warps=warps)
     p.prefill(prompts, max(prompts))
     p.check_ring()
     B = 5
@@ -419,12 +427,13 @@ def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out):
     p.close()
 
 
+@pytest.mark.parametrize("warps", [0, 3])
 @pytest.mark.parametrize("W,E,prompts", [(150, 1, [0, 70, 149]), (300, 75, [64, 0, 130])])
-def test_head_dim_64_tensor_core_attention_with_pinned_prompt(W, E, prompts):
+def test_head_dim_64_tensor_core_attention_with_pinned_prompt(warps, W, E, prompts):
     """The D = 64 variant of the TMA attention kernel (64-token tiles), several tiles, pinned entries that end inside
     a tile, group size 7."""
     p = Pair(pt, n_layers=2, batch=3, n_q_heads=14, n_kv_heads=2, head_dim=64, window=W, evict_chunk=E, dtype="bf16",
-             seed=W + 1, n_global=16, rank=16)
+             seed=W + 1, n_global=16, rank=16, attn_consumer_warps=warps)
     assert p.cache.info()["tensor_core_attn"]
     p.prefill(prompts, max(prompts))
     for t in range(W + 2 * E + 30):
@@ -510,3 +519,57 @@ def test_sequences_finish_and_their_places_are_reused(dtype, E):
     p.check_state()
     assert p.cache.status() == 0
     p.close()
+
+
+def test_reset_clears_stale_split_unit_counters_and_status():
+    """A launch that gives up part-way can leave arrival counts of split units behind.  Stand-in for that (no fault
+    is provoked): non-zero counters and a status word are written into the workspace by hand; after the full reset
+    attention over freshly filled rings is right again -- with stale counters the last-arriver test of a split unit
+    would fire early or never."""
+    p = Pair(pt, n_layers=2, batch=7, n_q_heads=28, n_kv_heads=4, head_dim=128, window=700, dtype="bf16", seed=33)
+    ptr_t, n_t = p.cache.workspace_region(pt.binding.REGION_TICKETS)
+    ptr_s, n_s = p.cache.workspace_region(pt.binding.REGION_STATUS)
+    base = p.cache.workspace.data_ptr()
+    tickets = p.cache.workspace[ptr_t - base: ptr_t - base + n_t].view(torch.int32)
+    status = p.cache.workspace[ptr_s - base: ptr_s - base + n_s].view(torch.int32)
+    assert tickets.numel() == 2 * 7 * 4 and int(tickets.abs().max()) == 0
+    tickets.copy_(torch.arange(1, tickets.numel() + 1, dtype=torch.int32, device="cuda") % 3 + 1)
+    status.fill_(1)
+    assert p.cache.status() == 1
+    p.cache.reset()
+    p.orc.reset()
+    assert p.cache.status() == 0 and int(tickets.abs().max()) == 0
+    for t in range(700 + 5):
+        if t in (0, 31, 32, 699, 700, 704):
+            p.step(t)
+        else:
+            q = p.gen.step_q(t)
+            k, v = p.gen.step_kv(t)
+            p.cache.decode_step(-1, q, k, v, p.out)
+            for l in range(2):
+                p.orc.append_evict(l, np64(k[l]), np64(v[l]))
+                p.orc.encode(l)
+    assert int(tickets.abs().max()) == 0            # the counters clean themselves after every launch
+    p.check_ring(); p.check_state()
+    assert p.cache.status() == 0
+    p.close()
+
+
+def test_launch_info_reports_the_instantiation():
+    """Three consumer warps on long launches of long windows, four otherwise; the configuration can fix either."""
+    c7 = dict(CONFIGS["qwen7b"])
+    kw = dict(n_q_heads=c7["n_q_heads"], n_kv_heads=c7["n_kv_heads"], head_dim=128, dtype="bf16")
+    small = pt.Cache(pt.make_config(n_layers=2, batch=2, window=2048, **kw))
+    assert small.attn_launch_info(-1) == {"consumer_warps": 4, "tile_tokens": 32, "stages": 12}
+    small.close()
+    forced = pt.Cache(pt.make_config(n_layers=2, batch=2, window=2048, attn_consumer_warps=3, **kw))
+    assert forced.attn_launch_info(-1)["consumer_warps"] == 3 and forced.attn_launch_info(0)["consumer_warps"] == 3
+    forced.close()
+    full = pt.Cache(pt.make_config(n_layers=28, batch=128, window=2048, **kw))      # the 7B-shaped workload
+    assert full.attn_launch_info(-1)["consumer_warps"] == 3          # 917,504 tiles of 64 per unit
+    assert full.attn_launch_info(0)["consumer_warps"] == 4           # one layer alone is a short launch
+    full.close()
+    torch.cuda.empty_cache()
+    gen = pt.Cache(pt.make_config(n_layers=1, batch=2, n_q_heads=4, n_kv_heads=1, head_dim=64, window=64, dtype="fp32"))
+    assert gen.attn_launch_info(-1) == {"consumer_warps": 0, "tile_tokens": 0, "stages": 0}
+    gen.close()
