@@ -5,7 +5,8 @@ One "step" = one decode step of the whole batch over all L layers, through ptenc
 steady state: every ring full, every sequence evicting one token per step.  Workload at 1 GPU = the
 Qwen2.5-7B-shaped configuration the metric is quoted on; other workloads with --workload.
 
-    python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
+    python bench.py --gpus N --steps K --warmup W            (N > 1: under torch.distributed.run, or run directly,
+                                                              in which case the script starts the N ranks itself)
     python bench.py --impl reference ...                     (times the CPU oracle on a bounded sample)
 
 Prints ONE JSON line on rank 0.
@@ -24,6 +25,40 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+
+def _oracle_worker(path: str) -> None:
+    """One process of the CPU-oracle timing: loads its inputs (numpy arrays written by the parent), builds the
+    oracle's cache for one layer, fills the window, says "ready", waits for "go" on stdin, runs the timed steps and
+    prints the seconds they took.  Imports numpy and the oracle only, so that many of these start quickly."""
+    import numpy as np
+    from oracle.ptenc_oracle import OracleCache
+    d = np.load(path, allow_pickle=False)
+    n_seq, W, E, n_prompt = int(d["n_seq"]), int(d["window"]), int(d["evict_chunk"]), int(d["n_prompt"])
+    orc = OracleCache(n_layers=1, batch=n_seq, n_q_heads=int(d["n_q_heads"]), n_kv_heads=int(d["n_kv_heads"]),
+                      head_dim=int(d["head_dim"]), window=W, evict_chunk=E, n_global=int(d["n_global"]),
+                      rank=int(d["rank"]))
+    orc.set_encoder(0, **{k: d["enc_" + k] for k in ("Wq_a", "Wk_a", "Wv_a", "q_g", "k_g", "v_g")})
+    q, k, v = d["q"], d["k"], d["v"]                      # [R, n_seq, H, D] each
+    R = q.shape[0]
+    if n_prompt > 0:
+        orc.prefill(0, d["Kp"], d["Vp"], [n_prompt] * n_seq)
+    for t in range(W - n_prompt):                         # fill (not timed)
+        orc.append_evict(0, k[t % R], v[t % R])
+    for t in range(int(d["warm"])):
+        orc.decode_step(0, q[t % R], k[t % R], v[t % R])
+    print("ready", flush=True)
+    sys.stdin.readline()
+    n_steps = int(d["n_steps"])
+    w0, c0 = time.perf_counter(), time.process_time()
+    for t in range(n_steps):
+        orc.decode_step(0, q[t % R], k[t % R], v[t % R])
+    print(json.dumps({"wall": time.perf_counter() - w0, "cpu": time.process_time() - c0}), flush=True)
+
+
+if __name__ == "__main__" and len(sys.argv) == 3 and sys.argv[1] == "--oracle-worker":
+    _oracle_worker(sys.argv[2])
+    sys.exit(0)
+
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
@@ -33,7 +68,10 @@ METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0029   # (dram read + write) / algorithmic, ncu, see profiles/
+# DRAM bytes moved (read + written, ncu counters) per algorithmic byte of the tensor-core attention kernel, keyed by
+# window: each ratio was measured on a launch with a smaller batch of the same head shape and window, and DRAM
+# traffic grows in proportion to the K/V tiles a launch reads.  Windows with no capture report no traffic figure.
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2048: 1.0030}
 
 
 def workload_cfg(name: str) -> dict:
@@ -148,54 +186,109 @@ class ClockSampler:
 
 
 # ======================================================================================== CPU oracle legs
-def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, n_prompt: int = 0):
-    """Times the CPU oracle, as it stands, on 1 layer x n_seq sequences at the full window.
-    Returns (seconds per sampled step, threads used)."""
-    from oracle.ptenc_oracle import OracleCache
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, n_prompt: int = 0, workers: int = 1):
+    """Times the CPU oracle, as it stands, on `workers` processes at once, each holding 1 layer x n_seq sequences of
+    its own at the full window (sequences are independent, so this is how the oracle uses many cores).  Every
+    process runs single-threaded; all start their timed steps together.  Returns (seconds per sampled step = the
+    slowest process's, processes, cpu-seconds used per wall-second)."""
+    tmp = f"/tmp/ptenc_oracle_{os.getpid()}"
+    os.makedirs(tmp, exist_ok=True)
     cc = {**c, "n_layers": 1, "batch": n_seq}
-    gen = make_inputs(cc, seed=0, device="cpu")
-    orc = OracleCache(n_layers=1, batch=n_seq, n_q_heads=c["n_q_heads"], n_kv_heads=c["n_kv_heads"],
-                      head_dim=c["head_dim"], window=c["window"], evict_chunk=E, n_global=c["n_global"],
-                      rank=c["rank"])
-    P = gen.encoder_params(0)
-    orc.set_encoder(0, **{k: v.double().numpy() for k, v in P.items()})
-    pool = []
-    for t in range(4):
-        k, v = gen.step_kv(t)
-        pool.append((gen.step_q(t)[0].double().numpy(), k[0].double().numpy(), v[0].double().numpy()))
-    if n_prompt > 0:                                   # pinned prompt, as on the GPU side
-        Kp = gen.generic(50, 0, (1, n_seq, n_prompt, c["n_kv_heads"], c["head_dim"]), 1.0)[0].double().numpy()
-        Vp = gen.generic(51, 0, (1, n_seq, n_prompt, c["n_kv_heads"], c["head_dim"]), 1.0)[0].double().numpy()
-        orc.prefill(0, Kp, Vp, [n_prompt] * n_seq)
-    for t in range(c["window"] - n_prompt):                  # fill (not timed)
-        _, k, v = pool[t % 4]
-        orc.append_evict(0, k, v)
-    for t in range(warm):
-        orc.decode_step(0, *pool[t % 4])
-    w0, c0 = time.perf_counter(), time.process_time()
-    for t in range(n_steps):
-        orc.decode_step(0, *pool[t % 4])
-    wall = time.perf_counter() - w0
-    cpu = time.process_time() - c0
-    return wall / n_steps, max(1, int(round(cpu / wall)))
+    env = {**os.environ, "OMP_NUM_THREADS": "1", "OPENBLAS_NUM_THREADS": "1", "MKL_NUM_THREADS": "1"}
+    procs, paths = [], []
+    for w in range(workers):
+        gen = make_inputs(cc, seed=1000 + w, device="cpu")          # every process decodes its own sequences
+        P = gen.encoder_params(0)
+        R = 4
+        q = np.stack([gen.step_q(t)[0].double().numpy() for t in range(R)])
+        kv = [gen.step_kv(t) for t in range(R)]
+        arrays = dict(n_seq=n_seq, window=c["window"], evict_chunk=E, n_prompt=n_prompt, n_q_heads=c["n_q_heads"],
+                      n_kv_heads=c["n_kv_heads"], head_dim=c["head_dim"], n_global=c["n_global"], rank=c["rank"],
+                      warm=warm, n_steps=n_steps, q=q, k=np.stack([x[0][0].double().numpy() for x in kv]),
+                      v=np.stack([x[1][0].double().numpy() for x in kv]),
+                      **{"enc_" + k: v.double().numpy() for k, v in P.items()})
+        if n_prompt > 0:
+            shape = (1, n_seq, n_prompt, c["n_kv_heads"], c["head_dim"])
+            arrays["Kp"] = gen.generic(50, 0, shape, 1.0)[0].double().numpy()
+            arrays["Vp"] = gen.generic(51, 0, shape, 1.0)[0].double().numpy()
+        path = os.path.join(tmp, f"w{w}.npz")
+        np.savez(path, **arrays)
+        paths.append(path)
+        procs.append(subprocess.Popen([sys.executable, os.path.join(ROOT, "bench.py"), "--oracle-worker", path],
+                                      stdin=subprocess.PIPE, stdout=subprocess.PIPE, text=True, env=env, cwd=ROOT))
+    try:
+        for p in procs:
+            if p.stdout.readline().strip() != "ready":
+                raise RuntimeError("oracle worker failed to start")
+        for p in procs:
+            p.stdin.write("go\n")
+            p.stdin.flush()
+        res = [json.loads(p.stdout.readline()) for p in procs]
+    finally:
+        for p in procs:
+            try:
+                p.stdin.close()
+            except Exception:
+                pass
+            p.wait(timeout=60)
+        for path in paths:
+            try:
+                os.remove(path)
+            except OSError:
+                pass
+        try:
+            os.rmdir(tmp)
+        except OSError:
+            pass
+    wall = max(r["wall"] for r in res)
+    return wall / n_steps, workers, sum(r["cpu"] for r in res) / wall
+
+
+def oracle_baseline(c: dict, n_steps: int, E: int, n_prompt: int, warm: int = 1) -> dict:
+    """The oracle on one core and on all host cores; tokens/s normalised to all L layers."""
+    L, B, W = c["n_layers"], c["batch"], c["window"]
+    nproc = host_cores()
+    n1 = min(8, B)
+    sec1, _, busy1 = oracle_sample(c, n1, n_steps, warm=warm, E=E, n_prompt=n_prompt, workers=1)
+    nw = 2                                                   # sequences per process on the all-cores leg
+    secN, P, busyN = oracle_sample(c, nw, n_steps, warm=warm, E=E, n_prompt=n_prompt, workers=nproc)
+    return {
+        "value": P * nw / (secN * L), "unit": UNIT, "cores": P, "nproc": nproc, "kind": "oracle",
+        "cpu_seconds_per_wall_second": busyN,
+        "one_core": {"value": n1 / (sec1 * L), "unit": UNIT, "cores": 1, "cpu_seconds_per_wall_second": busy1,
+                     "seconds_per_sampled_step": sec1,
+                     "sample": f"1 process x {n1} of {B} sequences x 1 of {L} layers x {n_steps} steps"},
+        "seconds_per_sampled_step": secN,
+        "sample": (f"oracle decode_step, as it stands: {P} single-threaded processes (one per host core) x {nw} sequences "
+                   f"each x 1 of {L} layers x {n_steps} steps at window {W} (full, evicting), timed together; "
+                   f"tokens/s = sequences / (step time x {L} layers)"),
+    }
 
 
 def run_reference(args, c: dict):
     """--impl reference: the oracle on a bounded sample; tokens/s normalised to all L layers."""
     if rank_env()[0] != 0:
         return
-    n_seq = 8 if c["batch"] >= 8 else c["batch"]
-    sec, cores = oracle_sample(c, n_seq, max(1, args.steps), warm=max(1, args.warmup), E=args.evict_chunk, n_prompt=args.prompt_len)
-    value = n_seq / (sec * c["n_layers"])
-    sample = (f"1 of {c['n_layers']} layers x {n_seq} of {c['batch']} sequences per step at window {c['window']} "
-              f"(full, evicting); tokens/s = {n_seq} / (step time x {c['n_layers']} layers)")
+    base = oracle_baseline(c, max(1, args.steps), args.evict_chunk, args.prompt_len, warm=max(1, args.warmup))
+    L, B = c["n_layers"], c["batch"]
+    seqs = base["cores"] * 2
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * c["n_layers"] * c["batch"] / n_seq,
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        # measured: one sampled step = every process decoding one token for its sequences in one layer
+        "ms_per_step": base["seconds_per_sampled_step"] * 1e3,
+        "ms_per_full_step_extrapolated": base["seconds_per_sampled_step"] * 1e3 * L * B / seqs,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config_block(args, c),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
@@ -227,6 +320,48 @@ def rank_env():
     """(rank, world size, local rank) from the launcher's environment; (0, 1, 0) when run directly."""
     return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
             int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def launcher_argv(n_gpus: int, argv) -> list:
+    """The command that runs this script as n_gpus ranks on one node (one process per GPU, rendezvous on the loopback
+    address)."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"), *argv]
+
+
+def ensure_ranks(args) -> None:
+    """`--gpus N` with N > 1 needs N ranks.  Started by a launcher (WORLD_SIZE set) the two must agree; started
+    directly, the script starts the ranks itself and this process becomes the launcher."""
+    world = os.environ.get("WORLD_SIZE")
+    if world is not None:
+        if int(world) != args.gpus:
+            sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started {world} ranks")
+        return
+    if args.gpus > 1:
+        cmd = launcher_argv(args.gpus, sys.argv[1:])
+        os.execv(cmd[0], cmd)
+
+
+def run_dry(args, c: dict):
+    """--dry-run: the rank plumbing alone (process group on gloo, barrier, max over ranks, one line from rank 0), no
+    GPU and no kernels.  Not a measurement."""
+    rank, world, local = rank_env()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = max_over_ranks([float(rank + 1)], dist, "cpu")[0]
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "ranks_seen_max_ms": ms,
+                          "config": config_block(args, c)}), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
 
 
 def shard_seed(rank: int) -> int:
@@ -402,10 +537,8 @@ def run_gpu(args, c: dict):
         step_gbs = bm["step"] / (ms_total * 1e-3) / 1e9
         bm["attn"] /= K                                          # per launch / per step averages from here on
         bm["step"] /= K
-        # DRAM bytes per algorithmic byte of the attention kernel, from the ncu capture summarised in
-        # profiles/attn_bf16_and_step_e1_ncu_full_stress-w2048-b16.md (a smaller batch of the same shape; traffic grows in
-        # proportion to the tiles processed), scaled to this launch.
-        traffic = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE * bm["attn"] if c["dtype"] == "bf16" else None
+        ratio = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(W) if cache_info["tensor_core_attn"] and P == 0 else None
+        traffic = ratio * bm["attn"] if ratio is not None else None
         bm.pop("attn_per_step")
         line = {
             "metric": METRIC, "value": job_tokens_per_s(world, B, K, ms_total), "unit": UNIT, "n_gpus": world,
@@ -429,12 +562,7 @@ def run_gpu(args, c: dict):
             **({"extras": extras} if extras else {}),
         }
         if world == 1 and not args.no_cpu_baseline:
-            n_seq, n_steps = min(8, B), args.cpu_steps
-            sec, cores = oracle_sample(c, n_seq, n_steps, E=E, n_prompt=P)
-            line["cpu_baseline"] = {
-                "value": n_seq / (sec * L), "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": (f"oracle decode_step on 1 of {L} layers x {n_seq} of {B} sequences x {n_steps} steps at "
-                           f"window {W} (full, evicting); tokens/s = {n_seq} / (step time x {L} layers)")}
+            line["cpu_baseline"] = oracle_baseline(c, args.cpu_steps, E, P)
         print(json.dumps(line), flush=True)
     cache.close()
     if dist is not None:
@@ -457,8 +585,11 @@ def main():
     ap.add_argument("--prompt-len", type=int, default=0,
                     help="tokens of a pinned prompt per sequence (kept for the whole rollout; the window slides over "
                          "the remaining slots)")
-    ap.add_argument("--cpu-steps", type=int, default=128, help="steps of the CPU-oracle sample")
+    ap.add_argument("--cpu-steps", type=int, default=96, help="steps of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="exercise the launch and rank plumbing only (gloo, no GPU, no kernels); prints a line marked "
+                         "dry_run")
     ap.add_argument("--extras", action="store_true",
                     help="also time the encoder's burst on a staged chunk (with --evict-chunk > 1) and the dynamic "
                          "weight update, each alone")
@@ -468,6 +599,10 @@ def main():
         c["n_global"] = args.n_global
     if args.impl == "reference":
         run_reference(args, c)
+        return
+    ensure_ranks(args)
+    if args.dry_run:
+        run_dry(args, c)
         return
     if args.warmup < 3:
         args.warmup = 3

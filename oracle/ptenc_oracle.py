@@ -7,8 +7,9 @@ only by the tests, by the smoke check and by the benchmark's CPU-baseline leg.
 What follows which passage
 --------------------------
 * cache bookkeeping  : Sec. 3.1 (the cache grows by one entry per decoded token),
-  Sec. 3.2 (a cache policy D prunes the context at every step), Sec. 3.3 ("until
-  the KV cache is full ... earlier tokens are evicted"; sliding-window policy),
+  Sec. 3.2 (a cache policy D prunes the context at every step), Sec. 3.3 (decoding
+  goes on while the cache has room, then the policy removes the oldest tokens;
+  sliding-window policy),
   Sec. 4.1 implementation details (a fraction of the tokens is evicted on
   saturation -> chunk size E).
 * attention          : the two unnumbered equations of Sec. 3.1:
@@ -41,6 +42,19 @@ in the tests where the mathematics allows):
   rollout, is attended by every later query, is never evicted and never encoded; the sliding
   window runs over the remaining W - n entries, and a chunk never exceeds that capacity.
 
+* importance-aware eviction (Sec. 4.3, the paragraph on inference-time token dropping: strategies
+  that account for token importance are plugged in where the sliding window drops tokens; the
+  paper names other systems and defines none of its own).  Reading taken, policy "score": a
+  token's importance is the attention mass it has received so far, summed over all query heads
+  of the layer (the softmax weights of Sec. 3.1, accumulated step by step; a token starts at
+  zero and first receives mass in the step it arrives).  When the cache is full, the tokens that
+  leave are the lowest-scoring ones among the candidates -- the unpinned tokens that are not
+  among the `recent` newest (the protection shrinks when the capacity leaves no other choice) --
+  ties going to the older token; they reach the encoder oldest first and their slots are reused
+  in that order.  The mass of the latest attention on a layer is folded into the scores when the
+  next token arrives on that layer, so repeating an attention call changes nothing.
+  -- parity unpinned for the choice of importance measure; the arithmetic is pinned.
+
 All arithmetic is float64.  Library primitives used as steps: numpy matmul, exp.
 """
 from __future__ import annotations
@@ -71,6 +85,21 @@ def attention_one_head(q, K, V):
     p = e / z
     o = p @ V
     return o, smax + np.log(z)
+
+
+def attention_mass(q, K):
+    """Attention mass each cached token receives from one decoded token: the softmax weights of Sec. 3.1 summed over
+    all query heads.  q [Hq, D]; K [n, Hkv, D].  Returns [n]; its entries sum to Hq."""
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    Hq, D = q.shape
+    g = Hq // K.shape[1]
+    mass = np.zeros((K.shape[0],), F64)
+    for h in range(Hq):
+        s = (K[:, h // g, :] @ q[h]) / np.sqrt(F64(D))
+        e = np.exp(s - np.max(s))
+        mass += e / np.sum(e)
+    return mass
 
 
 def attention_gqa(q, K, V):
@@ -171,14 +200,18 @@ class _Seq:
         self.K = np.zeros((W, Hkv, D), F64)
         self.V = np.zeros((W, Hkv, D), F64)
         self.n_appended = 0
+        self.score = {}                     # token index -> attention mass received so far (policy "score")
+        self.pending = None                 # (token list, mass) of the latest attention, not yet folded in
 
 
 class OracleCache:
     """Reference decode state for L layers x B sequences."""
 
     def __init__(self, *, n_layers, batch, n_q_heads, n_kv_heads, head_dim, window,
-                 evict_chunk=1, n_global=32, rank=32, normalize_mode=0, encode_enabled=1):
+                 evict_chunk=1, n_global=32, rank=32, normalize_mode=0, encode_enabled=1, policy="fifo", recent=0):
         assert n_q_heads % n_kv_heads == 0 and 1 <= evict_chunk <= window
+        assert policy in ("fifo", "score") and recent >= 0
+        self.policy, self.recent = policy, recent
         self.L, self.B = n_layers, batch
         self.Hq, self.Hkv, self.D = n_q_heads, n_kv_heads, head_dim
         self.W, self.E = window, evict_chunk
@@ -189,6 +222,7 @@ class OracleCache:
         self.S = [None] * n_layers          # [B, G, r]
         self.S0 = [None] * n_layers         # [G, r] initial state of the layer
         self.staged = [[None] * batch for _ in range(n_layers)]   # (K_e, V_e) of the last append
+        self.margin = [[np.inf] * batch for _ in range(n_layers)] # policy "score": see _evict_lowest_scores
 
     # -- set-up ------------------------------------------------------------------------
     def set_encoder(self, layer, Wq_a, Wk_a, Wv_a, q_g, k_g=None, v_g=None):
@@ -247,13 +281,20 @@ class OracleCache:
                 continue
             toks, sl = [], []
             capacity = self.W - len(c.pinned)       # entries the sliding part may hold
+            if c.pending is not None:               # mass of the latest attention on this layer joins the scores
+                for t_tok, m_tok in zip(*c.pending):
+                    c.score[t_tok] += m_tok
+                c.pending = None
             if len(c.live) == capacity:
-                for _ in range(min(self.E, capacity)):
-                    t_old = c.live.popleft()
-                    s_old = c.slot_of.pop(t_old)
-                    toks.append(t_old)
-                    sl.append(s_old)
-                    c.free.append(s_old)
+                if self.policy == "score":
+                    toks, sl = self._evict_lowest_scores(layer, b, capacity)
+                else:
+                    for _ in range(min(self.E, capacity)):
+                        t_old = c.live.popleft()
+                        s_old = c.slot_of.pop(t_old)
+                        toks.append(t_old)
+                        sl.append(s_old)
+                        c.free.append(s_old)
                 Ke = np.stack([c.K[s].reshape(-1) for s in sl])   # [m, d_kv], age order
                 Ve = np.stack([c.V[s].reshape(-1) for s in sl])
                 self.staged[layer][b] = (Ke, Ve)
@@ -264,10 +305,43 @@ class OracleCache:
             c.live.append(t)
             c.slot_of[t] = s_new
             c.n_appended = t + 1
+            if self.policy == "score":
+                c.score[t] = 0.0
             slots[b] = s_new
             ev_tokens.append(toks)
             ev_slots.append(sl)
         return slots, ev_tokens, ev_slots
+
+    def _evict_lowest_scores(self, layer, b, capacity):
+        """Policy "score": of the candidates (unpinned tokens other than the `recent` newest) the m lowest-scoring
+        leave, ties to the older token.  Returns (tokens, slots) oldest first and records the margin between the
+        highest score that left and the lowest candidate score that stayed."""
+        c = self.seqs[layer][b]
+        m = min(self.E, capacity)
+        protected = min(self.recent, capacity - m)
+        candidates = list(c.live)[:capacity - protected]              # arrival order; the newest are protected
+        chosen = sorted(candidates, key=lambda tok: (c.score[tok], tok))[:m]
+        left = set(chosen)
+        stayed = [c.score[tok] for tok in candidates if tok not in left]
+        self.margin[layer][b] = (min(stayed) - max(c.score[tok] for tok in chosen)) if stayed else np.inf
+        toks, sl = [], []
+        for t_old in sorted(chosen):                                  # they leave oldest first
+            c.live.remove(t_old)
+            s_old = c.slot_of.pop(t_old)
+            del c.score[t_old]
+            toks.append(t_old)
+            sl.append(s_old)
+            c.free.append(s_old)
+        return toks, sl
+
+    def scores(self, layer, b):
+        """{token: attention mass received so far}, the latest attention included, for the unpinned live tokens."""
+        c = self.seqs[layer][b]
+        out = dict(c.score)
+        if c.pending is not None:
+            for t_tok, m_tok in zip(*c.pending):
+                out[t_tok] += m_tok
+        return out
 
     # -- a3: encode -----------------------------------------------------------------------
     def encode(self, layer, K_e=None, V_e=None):
@@ -303,6 +377,9 @@ class OracleCache:
                 continue
             sl = [c.slot_of[t] for t in c.pinned] + [c.slot_of[t] for t in c.live]
             o[b], lse[b] = attention_gqa(q[b], c.K[sl], c.V[sl])
+            if self.policy == "score":
+                mass = attention_mass(q[b], c.K[sl])
+                c.pending = (list(c.live), mass[len(c.pinned):])      # pinned tokens are never candidates
         return o, lse
 
     # -- a4: one whole step for one layer --------------------------------------------------------

@@ -88,3 +88,23 @@ def test_reference_arm_under_a_two_rank_launch_prints_once():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["gpu_launches"] == 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
+
+
+def test_gpus_flag_without_a_launcher_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` run directly (no launcher environment) must not quietly run one rank: it re-executes
+    itself under the launcher.  Checked with the plumbing-only mode (gloo, no GPU): rank 0 reports two ranks."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR",
+                                                              "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--workload", "tiny"],
+                       capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(ln) for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1 and lines[0]["dry_run"] and lines[0]["n_gpus"] == 2 and lines[0]["ranks_seen_max_ms"] == 2.0
+    assert lines[0]["config"]["parallelism"].startswith("dp2")
+
+
+def test_gpus_flag_that_disagrees_with_the_launcher_is_an_error():
+    env = {**os.environ, "WORLD_SIZE": "1", "RANK": "0", "LOCAL_RANK": "0"}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--dry-run", "--workload", "tiny"],
+                       capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
+    assert r.returncode != 0 and "launcher started 1 ranks" in r.stderr

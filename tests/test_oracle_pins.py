@@ -380,7 +380,6 @@ def pin_encode_recurrence(mod):
         if t >= 2:
             np.testing.assert_allclose(c.S[0][0], S1 / np.linalg.norm(S1, axis=1, keepdims=True), atol=1e-12)
     # (f) modes 1 and 2
-    st1 = run(normalize_mode=None) if False else None
     c1 = _mk(mod, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, n_global=G, rank=r, window=W, normalize_mode=1)
     c2 = _mk(mod, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, n_global=G, rank=r, window=W, normalize_mode=2)
     c1.set_encoder(0, **P)
@@ -537,7 +536,168 @@ def pin_reset_gives_a_fresh_sequence(mod):
         assert np.array_equal(a.S[0][0], fresh.S[0][0])
 
 
-PINS = [pin_ring_closed_form, pin_ring_vs_list_model, pin_attention_full_window_is_causal,
+# ---------------------------------------------------------------- importance-aware eviction (Sec. 4.3 token dropping)
+def _score_cfg(mod, W, E, recent, **kw):
+    return _mk(mod, window=W, evict_chunk=E, policy="score", recent=recent, **kw)
+
+
+def pin_score_hand_worked(mod):
+    """Hq = Hkv = 1, D = 1, all queries zero, so every softmax is uniform and the masses are dyadic fractions.
+    W = 2, E = 1, nothing protected: token 0 collects 1, then 1/2 per step; every later token has 1/2 when the next
+    one arrives and is the one that leaves -- from its slot 1, which the newcomer takes.  With the newest token
+    protected the only candidate is the oldest: plain FIFO."""
+    c = _score_cfg(mod, 2, 1, 0, n_q_heads=1, n_kv_heads=1, head_dim=1, batch=1)
+    q0 = np.zeros((1, 1, 1))
+    left, slots = [], []
+    for t in range(6):
+        x = np.full((1, 1, 1), float(t + 1))
+        _, _, (sl, ev_t, ev_s) = c.decode_step(0, q0, x, x)
+        left.append(ev_t[0]); slots.append(int(sl[0]))
+    assert left == [[], [], [1], [2], [3], [4]] and slots == [0, 1, 1, 1, 1, 1]
+    assert c.scores(0, 0) == {0: 1.0 + 5 * 0.5, 5: 0.5}
+    assert c.margin[0][0] == (1.0 + 4 * 0.5) - 0.5              # token 0 stayed with 3.0 when token 4 left with 0.5
+    f = _score_cfg(mod, 2, 1, 1, n_q_heads=1, n_kv_heads=1, head_dim=1, batch=1)
+    left = []
+    for t in range(6):
+        x = np.full((1, 1, 1), float(t + 1))
+        left.append(f.decode_step(0, q0, x, x)[2][1][0])
+    assert left == [[], [], [0], [1], [2], [3]]
+
+
+def _naive_score_rollout(W, E, recent, n_prompt, q, kk, vv, Hq, Hkv):
+    """Independent model.  Rows of kk, vv are the tokens in arrival order, the first n_prompt of them a pinned
+    prompt.  The whole history is kept; the scores at an eviction are recomputed from scratch as the sum, over every
+    earlier step, of the torch softmax weights that step's query gave the token."""
+    g = Hq // Hkv
+    T, D = q.shape[0], q.shape[-1]
+    live = list(range(n_prompt))
+    attn_hist, evicted_hist, live_hist, out_hist, score_hist = [], [], [], [], []
+    for t in range(T):
+        tok = n_prompt + t
+        sliding = [x for x in live if x >= n_prompt]
+        cap = W - n_prompt
+        ev = []
+        if len(sliding) == cap:
+            m = min(E, cap)
+            prot = min(recent, cap - m)
+            cand = sorted(sliding)[:cap - prot]
+            sc = np.array([sum(mass[lst.index(x)] for lst, mass in attn_hist if x in lst) for x in cand])
+            order = np.lexsort((np.array(cand), sc))          # by score, then by token index
+            ev = sorted(cand[i] for i in order[:m])
+            live = [x for x in live if x not in ev]
+        live.append(tok)
+        K = torch.tensor(np.stack([kk[x] for x in live]))     # [n, Hkv, D]
+        V = torch.tensor(np.stack([vv[x] for x in live]))
+        mass = np.zeros(len(live))
+        o = np.zeros((Hq, D))
+        for h in range(Hq):
+            w = torch.softmax(K[:, h // g] @ torch.tensor(q[t, h]) / np.sqrt(D), dim=0)
+            mass += w.numpy()
+            o[h] = (w @ V[:, h // g]).numpy()
+        attn_hist.append((list(live), mass))
+        evicted_hist.append(ev); live_hist.append(list(live)); out_hist.append(o)
+        score_hist.append({x: sum(ms[lst.index(x)] for lst, ms in attn_hist if x in lst) for x in live if x >= n_prompt})
+    return evicted_hist, live_hist, out_hist, score_hist
+
+
+def pin_score_policy_vs_brute_force(mod):
+    rng = np.random.default_rng(77)
+    Hq, Hkv, D = 4, 2, 4
+    for W, E, recent, n_prompt in [(4, 1, 0, 0), (6, 2, 1, 0), (9, 3, 3, 2), (5, 5, 0, 0), (7, 2, 4, 3), (6, 1, 5, 0)]:
+        T = 40
+        q = rng.standard_normal((T, Hq, D)) * 2
+        k = rng.standard_normal((T, Hkv, D))
+        v = rng.standard_normal((T, Hkv, D))
+        kp = rng.standard_normal((n_prompt, Hkv, D))
+        vp = rng.standard_normal((n_prompt, Hkv, D))
+        c = _score_cfg(mod, W, E, recent, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D)
+        if n_prompt:
+            c.prefill(0, kp[None], vp[None], [n_prompt])
+        ev_want, live_want, out_want, score_want = _naive_score_rollout(
+            W, E, recent, n_prompt, q, np.concatenate([kp, k]), np.concatenate([vp, v]), Hq, Hkv)
+        n_ev = 0
+        for t in range(T):
+            o, _, (sl, ev_t, ev_s) = c.decode_step(0, q[t][None], k[t][None], v[t][None])
+            assert ev_t[0] == ev_want[t], (W, E, recent, n_prompt, t, ev_t[0], ev_want[t])
+            assert sorted(list(c.seqs[0][0].pinned) + list(c.seqs[0][0].live)) == sorted(live_want[t])
+            np.testing.assert_allclose(o[0], out_want[t], atol=1e-12)
+            got = c.scores(0, 0)
+            assert set(got) == set(score_want[t])
+            for tok, val in score_want[t].items():
+                assert abs(got[tok] - val) < 1e-12, (W, E, recent, n_prompt, t, tok)
+            assert len(c.seqs[0][0].live) + n_prompt <= W
+            n_ev += len(ev_t[0])
+        assert n_ev >= T - W - 1
+        # not the sliding window: some token outlived W later arrivals (except where everything is protected)
+        if recent < W - n_prompt - min(E, W - n_prompt):
+            assert min(c.seqs[0][0].live) < n_prompt + T - W
+
+
+def pin_score_policy_reduces_to_fifo(mod):
+    """(a) No attention is ever run, so every score is zero and every tie goes to the older token: the sliding window.
+    (b) Everything but the E oldest tokens is protected: the candidates are exactly the tokens FIFO evicts, whatever
+    the scores, and outputs, slots and states equal the sliding-window cache's."""
+    rng = np.random.default_rng(5)
+    for W, E in [(3, 1), (6, 2), (8, 8), (7, 3)]:
+        a = _score_cfg(mod, W, E, 0, batch=2)
+        f = _mk(mod, window=W, evict_chunk=E, batch=2)
+        for t in range(4 * W + 3):
+            x = rng.standard_normal((2, 1, 4))
+            ra, rf = a.append_evict(0, x, x), f.append_evict(0, x, x)
+            assert list(ra[0]) == list(rf[0]) and ra[1] == rf[1] and ra[2] == rf[2], (W, E, t)
+        enc = dict(Wq_a=rng.standard_normal((2, 8)), Wk_a=rng.standard_normal((2, 4)), Wv_a=rng.standard_normal((2, 4)),
+                   q_g=rng.standard_normal((3, 8)), k_g=rng.standard_normal((3, 4)), v_g=rng.standard_normal((3, 4)))
+        b = _score_cfg(mod, W, E, W - E, batch=2)
+        f = _mk(mod, window=W, evict_chunk=E, batch=2)
+        b.set_encoder(0, **enc); f.set_encoder(0, **enc)
+        for t in range(4 * W + 3):
+            q, x, y = rng.standard_normal((2, 2, 4)), rng.standard_normal((2, 1, 4)), rng.standard_normal((2, 1, 4))
+            ob, lb_, rb = b.decode_step(0, q, x, y)
+            of, lf_, rf = f.decode_step(0, q, x, y)
+            assert list(rb[0]) == list(rf[0]) and rb[1] == rf[1] and rb[2] == rf[2]
+            assert np.array_equal(ob, of) and np.array_equal(b.S[0], f.S[0])
+
+
+def pin_score_mass_bookkeeping(mod):
+    """Every decoded token hands out exactly Hq units of mass; what the live tokens hold plus what evicted tokens took
+    with them is Hq per step (no prompt).  Repeating the attention call changes nothing.  A token that draws almost
+    all the attention of every step is never evicted, while the sliding window drops it after W steps."""
+    rng = np.random.default_rng(9)
+    Hq, Hkv, D, W, E = 4, 2, 4, 5, 2
+    c = _score_cfg(mod, W, E, 1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D)
+    d = _score_cfg(mod, W, E, 1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D)
+    carried = 0.0
+    for t in range(30):
+        q, x = rng.standard_normal((1, Hq, D)), rng.standard_normal((1, Hkv, D))
+        before = c.scores(0, 0)
+        _, _, (sl, ev_t, ev_s) = c.decode_step(0, q, x, x)
+        carried += sum(before[tok] for tok in ev_t[0])
+        assert abs(sum(c.scores(0, 0).values()) + carried - Hq * (t + 1)) < 1e-9
+        assert set(c.scores(0, 0)) == set(c.seqs[0][0].live)
+        _, _, rec = d.decode_step(0, q, x, x)
+        d.decode_attn(0, q); d.decode_attn(0, rng.standard_normal((1, Hq, D))); d.decode_attn(0, q)
+        assert rec[1] == ev_t
+    assert c.scores(0, 0) == d.scores(0, 0)
+    total = sum(c.scores(0, 0).values())
+    for _ in range(3):                          # tokens arriving with no attention in between: nothing is added twice
+        before = c.scores(0, 0)
+        _, ev_t, _ = c.append_evict(0, x, x)
+        total -= sum(before[tok] for tok in ev_t[0])
+        assert abs(sum(c.scores(0, 0).values()) - total) < 1e-9
+    big = np.zeros((1, Hkv, D)); big[:, :, 0] = 8.0
+    s = _score_cfg(mod, 4, 1, 0, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D)
+    f = _mk(mod, window=4, evict_chunk=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D)
+    qq = np.zeros((1, Hq, D)); qq[:, :, 0] = 8.0
+    for t in range(40):
+        x = big if t == 0 else rng.standard_normal((1, Hkv, D)) * 0.1
+        s.decode_step(0, qq, x, x); f.decode_step(0, qq, x, x)
+        assert 0 in s.seqs[0][0].live
+    assert 0 not in f.seqs[0][0].live
+    assert s.scores(0, 0)[0] > 0.99 * Hq * 40
+
+
+PINS = [pin_score_hand_worked, pin_score_policy_vs_brute_force, pin_score_policy_reduces_to_fifo,
+        pin_score_mass_bookkeeping, pin_ring_closed_form, pin_ring_vs_list_model, pin_attention_full_window_is_causal,
         pin_attention_sliding_window, pin_attention_chunked_window, pin_attention_window_one,
         pin_attention_special_cases, pin_attention_gqa_mapping, pin_encode_worked_example,
         pin_encode_exact_rational, pin_encode_identities, pin_encode_recurrence,
@@ -592,6 +752,22 @@ MUTATIONS = {
     "lora_replaces_output": ("y[b] = y[b] + lora_delta(A, S[b], Bm) @ x[b]", "y[b] = lora_delta(A, S[b], Bm) @ x[b]"),
     "lora_shared_state": ("y[b] = y[b] + lora_delta(A, S[b], Bm) @ x[b]", "y[b] = y[b] + lora_delta(A, S[0], Bm) @ x[b]"),
     "lse_without_max": ("return o, smax + np.log(z)", "return o, np.log(z)"),
+    "score_ties_to_newer": ("key=lambda tok: (c.score[tok], tok))[:m]", "key=lambda tok: (c.score[tok], -tok))[:m]"),
+    "score_evicts_highest": ("key=lambda tok: (c.score[tok], tok))[:m]", "key=lambda tok: (-c.score[tok], tok))[:m]"),
+    "score_ignores_recent": ("protected = min(self.recent, capacity - m)", "protected = 0"),
+    "score_protection_blocks_eviction": ("protected = min(self.recent, capacity - m)", "protected = min(self.recent, capacity - 1)"),
+    "score_first_head_only": ("    for h in range(Hq):\n        s = (K[:, h // g, :] @ q[h]) / np.sqrt(F64(D))",
+                              "    for h in range(1):\n        s = (K[:, h // g, :] @ q[h]) / np.sqrt(F64(D))"),
+    "score_unnormalised_mass": ("        mass += e / np.sum(e)", "        mass += e"),
+    "score_mass_without_scale": ("s = (K[:, h // g, :] @ q[h]) / np.sqrt(F64(D))\n        e = np.exp(s - np.max(s))\n        mass",
+                                 "s = (K[:, h // g, :] @ q[h])\n        e = np.exp(s - np.max(s))\n        mass"),
+    "score_leave_in_score_order": ("for t_old in sorted(chosen):", "for t_old in chosen:"),
+    "score_folded_twice": ("                    c.score[t_tok] += m_tok\n                c.pending = None",
+                           "                    c.score[t_tok] += m_tok"),
+    "score_new_token_gets_no_mass": ("c.pending = (list(c.live), mass[len(c.pinned):])",
+                                     "c.pending = (list(c.live)[:-1], mass[len(c.pinned):-1])"),
+    "score_pinned_offset_forgotten": ("c.pending = (list(c.live), mass[len(c.pinned):])",
+                                      "c.pending = (list(c.live), mass[:len(c.live)])"),
 }
 
 
