@@ -93,7 +93,9 @@ typedef struct {
 /* Bytes of device workspace a cache with this configuration needs.  Host only, launches nothing.
  * Layout (all inside the workspace): K and V rings [L][B][H_kv][W][D]; ring state head/count (int32)
  * and n_appended (int64) [L][B], pinned-entry counts (int32) [L][B]; evicted-row staging [L][B][E][H_kv*D] for K and for V; state S
- * [L][B][G][r] fp32; per layer Q_a [G][r] fp32 and copies of W^a_K, W^a_V; split-K partials; status. */
+ * [L][B][G][r] fp32; per layer Q_a [G][r] fp32 and copies of W^a_K, W^a_V; split-K partials; status.  Under
+ * PTENC_POLICY_SCORE also per-slot scores and token indices, a liveness bitmap, the freed-slot queue, and the logits
+ * of the latest attention launch [L][B][H_kv][W][8] fp32 (6 % of the rings at head_dim 128). */
 PTENC_API int ptenc_workspace_bytes(const ptenc_config* cfg /*host*/, size_t* bytes /*host, out*/);
 
 /* Binds a cache to `dev_workspace` (1024-byte aligned, >= ptenc_workspace_bytes) and zeroes it on
@@ -206,6 +208,29 @@ PTENC_API int ptenc_get_ring(ptenc_cache* c, int layer, int32_t* head, int32_t* 
 
 /* Copies one layer's state to S_out [B, G, r] fp32 (device). */
 PTENC_API int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* stream);
+
+/* Importance-aware eviction, PTENC_POLICY_SCORE (Sec. 4.3, integration with inference-time token dropping; the paper
+ * plugs in strategies that account for token importance and leaves their efficient integration open -- the measure
+ * used here is this library's reading, stated below).
+ *
+ * A token's score is the attention mass it has received so far: the softmax weights of Sec. 3.1 that every query
+ * head of the layer gave it, summed over the heads and over the decode steps since it arrived.  When a token arrives
+ * at a full cache, the tokens that leave are the E lowest-scoring candidates -- the unpinned tokens other than the
+ * `recent` newest ones (fewer are protected when the capacity leaves no room) -- ties going to the older token.  They
+ * are staged for ptenc_encode oldest first, their slots are reused in that order, and everything downstream (a3,
+ * a2, the fused step) works as under the sliding window.  Slots are no longer a ring: ptenc_get_ring reports head 0.
+ * The mass of the latest attention launch on a layer (ptenc_decode_attn or the attention inside ptenc_decode_step) is
+ * folded into the scores when the next token arrives on that layer, so repeating an attention call changes nothing.
+ * Shapes: bf16, head_dim 64 or 128, n_q_heads/n_kv_heads <= 8, window <= 8192 (PTENC_ESHAPE otherwise).
+ *
+ * ptenc_get_evicted: tokens [B][E] (int64, oldest first), slots [B][E], n_evicted [B] of the last append on `layer`;
+ * entries past n_evicted[b] are stale.  ptenc_get_scores: score_out [B][W] fp32 and token_out [B][W] (token index
+ * held by each slot, -1 for free and pinned slots) as they stand, i.e. without the mass of an attention launch that
+ * has not been folded in yet.  Device pointers, each nullable in ptenc_get_evicted.  PTENC_EINVAL under
+ * PTENC_POLICY_FIFO. */
+PTENC_API int ptenc_get_evicted(ptenc_cache* c, int layer, int64_t* tokens, int32_t* slots, int32_t* n_evicted,
+                                void* stream);
+PTENC_API int ptenc_get_scores(ptenc_cache* c, int layer, float* score_out, int32_t* token_out, void* stream);
 
 /* Synchronises the device and reads the status word into *dev_status (host).  Returns PTENC_OK when it
  * is zero, PTENC_EDEVICE_STATUS otherwise.  The word is sticky until ptenc_cache_reset(c, NULL, ..). */

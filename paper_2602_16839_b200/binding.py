@@ -26,7 +26,7 @@ POLICY_FIFO, POLICY_SCORE = 0, 1
 EXPORTS = ["ptenc_workspace_bytes", "ptenc_cache_create", "ptenc_cache_destroy", "ptenc_cache_reset",
            "ptenc_set_encoder", "ptenc_prefill", "ptenc_get_pinned", "ptenc_append_evict", "ptenc_decode_attn", "ptenc_encode", "ptenc_lora_apply", "ptenc_decode_step",
            "ptenc_host_staging_bytes", "ptenc_decode_step_host",
-           "ptenc_get_ring", "ptenc_get_state", "ptenc_cache_status", "ptenc_cache_info", "ptenc_attn_launch_info",
+           "ptenc_get_ring", "ptenc_get_state", "ptenc_get_evicted", "ptenc_get_scores", "ptenc_cache_status", "ptenc_cache_info", "ptenc_attn_launch_info",
            "ptenc_workspace_region", "ptenc_time_next_attn", "ptenc_attn_rings_static", "ptenc_launch_count",
            "ptenc_strerror"]
 
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.ptenc_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u64, vp]
     lib.ptenc_get_ring.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ptenc_get_state.argtypes = [vp, i32, vp, vp]
+    lib.ptenc_get_evicted.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.ptenc_get_scores.argtypes = [vp, i32, vp, vp, vp]
     lib.ptenc_cache_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     lib.ptenc_cache_info.argtypes = [vp] + [ctypes.POINTER(ctypes.c_int32)] * 3
     lib.ptenc_attn_launch_info.argtypes = [vp, i32] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -223,6 +225,23 @@ class Cache:
         S = torch.empty(self.cfg.batch, self.cfg.n_global, self.cfg.rank, dtype=torch.float32, device=self.device)
         _check(lib.ptenc_get_state(self._h, layer, _ptr(S), _stream()), "ptenc_get_state")
         return S
+
+    def get_evicted(self, layer):
+        """(tokens [B, E] int64 oldest first, slots [B, E] int32, n_evicted [B] int32) of the last append (score policy)."""
+        B, E = self.cfg.batch, self.cfg.evict_chunk
+        tok = torch.full((B, E), -1, dtype=torch.int64, device=self.device)
+        slot = torch.full((B, E), -1, dtype=torch.int32, device=self.device)
+        n = torch.zeros(B, dtype=torch.int32, device=self.device)
+        _check(lib.ptenc_get_evicted(self._h, layer, _ptr(tok), _ptr(slot), _ptr(n), _stream()), "ptenc_get_evicted")
+        return tok, slot, n
+
+    def get_scores(self, layer):
+        """(score [B, W] fp32, token [B, W] int32, -1 where the slot holds no unpinned token) (score policy)."""
+        B, W = self.cfg.batch, self.cfg.window
+        score = torch.empty(B, W, dtype=torch.float32, device=self.device)
+        token = torch.empty(B, W, dtype=torch.int32, device=self.device)
+        _check(lib.ptenc_get_scores(self._h, layer, _ptr(score), _ptr(token), _stream()), "ptenc_get_scores")
+        return score, token
 
     def status(self) -> int:
         st = ctypes.c_int32(0)

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libptenc.so")
-SOURCES = ["ptenc_api.cu", "ptenc_ring.cu", "ptenc_encode.cu", "ptenc_encode_tc.cu", "ptenc_step_e1.cu", "ptenc_lora.cu", "ptenc_attn_generic.cu", "ptenc_attn_bf16.cu"]
+SOURCES = ["ptenc_api.cu", "ptenc_ring.cu", "ptenc_score.cu", "ptenc_encode.cu", "ptenc_encode_tc.cu", "ptenc_step_e1.cu", "ptenc_lora.cu", "ptenc_attn_generic.cu", "ptenc_attn_bf16.cu"]
 HEADERS = [os.path.join(CSRC, "ptenc_internal.h"), os.path.join(ROOT, "include", "ptenc.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]

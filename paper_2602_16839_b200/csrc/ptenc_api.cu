@@ -16,6 +16,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Layout {
   size_t K, V, head, count, n_app, n_sink, stageK, stageV, n_staged, evict_first, S, S0, Qa, Wk, Wv, enc_set,
       part_acc, part_ml, tickets, status, total;
+  // importance-aware policy only
+  size_t slot_tok, score, live_bits, logits, lse2, pending, fq, fq_head, fq_count, ev_tok, ev_slot;
 };
 
 int validate_config(const ptenc_config* c) {
@@ -29,8 +31,9 @@ int validate_config(const ptenc_config* c) {
   if (c->encode_enabled != 0 && c->encode_enabled != 1) return PTENC_EINVAL;
   if (c->device < 0) return PTENC_EINVAL;
   if (c->attn_consumer_warps != 0 && c->attn_consumer_warps != 3 && c->attn_consumer_warps != 4) return PTENC_EINVAL;
-  if (c->policy != PTENC_POLICY_FIFO) return PTENC_EINVAL;
-  if (c->recent != 0) return PTENC_EINVAL;
+  if (c->policy != PTENC_POLICY_FIFO && c->policy != PTENC_POLICY_SCORE) return PTENC_EINVAL;
+  if (c->recent < 0 || c->recent >= c->window) return PTENC_EINVAL;
+  if (c->policy == PTENC_POLICY_FIFO && c->recent != 0) return PTENC_EINVAL;
   if (c->n_q_heads % c->n_kv_heads != 0) return PTENC_ESHAPE;
   if (c->head_dim % 8 != 0 || c->head_dim > 256) return PTENC_ESHAPE;
   if (c->n_global < 1 || c->n_global > 128 || c->rank < 1 || c->rank > 128) return PTENC_ESHAPE;
@@ -38,6 +41,12 @@ int validate_config(const ptenc_config* c) {
   if ((long long)c->window > (1 << 24)) return PTENC_ESHAPE;
   const long long rows = (long long)c->n_layers * c->batch * c->n_kv_heads * c->window;
   if (rows >= (1ll << 31)) return PTENC_ESHAPE;
+  if (c->policy == PTENC_POLICY_SCORE) {
+    // the attention mass comes out of the tensor-core attention kernel; the selection sorts a window in shared memory
+    if (c->dtype != PTENC_DTYPE_BF16 || (c->head_dim != 64 && c->head_dim != 128) ||
+        c->n_q_heads / c->n_kv_heads > 8 || c->window > 8192)
+      return PTENC_ESHAPE;
+  }
   return PTENC_OK;
 }
 
@@ -68,6 +77,22 @@ Layout make_layout(const ptenc_config* c) {
   o.part_ml = take((size_t)PART_SLOTS * 16 * 4);
   o.tickets = take(L * B * Hkv * 4);
   o.status = take(64);
+  o.slot_tok = o.score = o.live_bits = o.logits = o.lse2 = o.pending = o.fq = o.fq_head = o.fq_count = o.ev_tok =
+      o.ev_slot = 0;
+  if (c->policy == PTENC_POLICY_SCORE) {
+    const size_t wb = (W + 63) / 64 * 2, Hq = c->n_q_heads;
+    o.slot_tok = take(L * B * W * 4);
+    o.score = take(L * B * W * 4);
+    o.live_bits = take(L * B * wb * 4);
+    o.logits = take(L * B * Hkv * W * 8 * 4);
+    o.lse2 = take(L * B * Hq * 4);
+    o.pending = take(L * B * 4);
+    o.fq = take(L * B * E * 4);
+    o.fq_head = take(L * B * 4);
+    o.fq_count = take(L * B * 4);
+    o.ev_tok = take(L * B * E * 8);
+    o.ev_slot = take(L * B * E * 4);
+  }
   o.total = off;
   return o;
 }
@@ -93,6 +118,29 @@ int check_layer(const ptenc_cache* c, int layer, int* l0, int* nl) {
   if (layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
   *l0 = layer; *nl = 1;
   return PTENC_OK;
+}
+
+// a1 under whichever eviction policy the cache was created with.
+cudaError_t launch_append(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new, const uint8_t* active,
+                          int32_t* slot_out, int64_t* evict_first_out, int32_t* n_evicted_out, cudaStream_t st) {
+  if (c->cfg.policy == PTENC_POLICY_SCORE)
+    return ptenc_launch_score_step(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out, st);
+  return ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out, st);
+}
+
+// a1 + a3 of a decode step: fused into one kernel in ring-per-step mode under the sliding-window policy, else the
+// append followed by the encode of the staged rows.
+bool launch_append_and_encode(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
+                              const uint8_t* active, cudaStream_t st, const char* who) {
+  (void)who;
+  if (c->cfg.policy == PTENC_POLICY_FIFO && c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0))
+    return ok(ptenc_launch_step_e1(c, l0, nl, true, k_new, v_new, active, nullptr, nullptr, nullptr, 0, st),
+              "decode_step/append_evict+encode", st);
+  if (!ok(launch_append(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st), "decode_step/append_evict", st))
+    return false;
+  if (c->cfg.encode_enabled)
+    return ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step/encode", st);
+  return true;
 }
 
 cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
@@ -196,6 +244,23 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   d.tickets = reinterpret_cast<int*>(base + lay.tickets);
   d.part_slots = PART_SLOTS;
   d.status = reinterpret_cast<int*>(base + lay.status);
+  d.policy = cfg->policy; d.recent = cfg->recent; d.wb = 0;
+  d.slot_tok = nullptr; d.score = nullptr; d.live_bits = nullptr; d.logits = nullptr; d.lse2 = nullptr;
+  d.pending = nullptr; d.fq = nullptr; d.fq_head = nullptr; d.fq_count = nullptr; d.ev_tok = nullptr; d.ev_slot = nullptr;
+  if (cfg->policy == PTENC_POLICY_SCORE) {
+    d.wb = (cfg->window + 63) / 64 * 2;
+    d.slot_tok = reinterpret_cast<int*>(base + lay.slot_tok);
+    d.score = reinterpret_cast<float*>(base + lay.score);
+    d.live_bits = reinterpret_cast<unsigned int*>(base + lay.live_bits);
+    d.logits = reinterpret_cast<float*>(base + lay.logits);
+    d.lse2 = reinterpret_cast<float*>(base + lay.lse2);
+    d.pending = reinterpret_cast<int*>(base + lay.pending);
+    d.fq = reinterpret_cast<int*>(base + lay.fq);
+    d.fq_head = reinterpret_cast<int*>(base + lay.fq_head);
+    d.fq_count = reinterpret_cast<int*>(base + lay.fq_count);
+    d.ev_tok = reinterpret_cast<long long*>(base + lay.ev_tok);
+    d.ev_slot = reinterpret_cast<int*>(base + lay.ev_slot);
+  }
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ws, 0, lay.total, st) != cudaSuccess) { delete c; return PTENC_ECUDA; }
@@ -269,8 +334,8 @@ int ptenc_append_evict(ptenc_cache* c, int layer, const void* k_new, const void*
   if (rc != PTENC_OK) return rc;
   if (k_new == nullptr || v_new == nullptr) return PTENC_EINVAL;
   if (misaligned(k_new) || misaligned(v_new)) return PTENC_EALIGN;
-  return ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out,
-                                   static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+  return launch_append(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out,
+                       static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* active, void* out, float* lse_out,
@@ -320,20 +385,7 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0)) {
-    // ring-per-step mode: append/evict and the encode of the evicted row in one kernel
-    if (!ok(ptenc_launch_step_e1(c, l0, nl, true, k_new, v_new, active, nullptr, nullptr, nullptr, 0, st),
-            "decode_step/append_evict+encode", st))
-      return PTENC_ECUDA;
-  } else {
-    if (!ok(ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st),
-            "decode_step/append_evict", st))
-      return PTENC_ECUDA;
-    if (c->cfg.encode_enabled) {
-      if (!ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step/encode", st))
-        return PTENC_ECUDA;
-    }
-  }
+  if (!launch_append_and_encode(c, l0, nl, k_new, v_new, active, st, "decode_step")) return PTENC_ECUDA;
   if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, st), "decode_step/attn", st)) return PTENC_ECUDA;
   return PTENC_OK;
 }
@@ -437,18 +489,7 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
   }
   // a1 + a3 on the caller's stream once the keys/values are on the device
   if (!good(cudaStreamWaitEvent(st, c->ev_kv, 0))) return PTENC_ECUDA;
-  if (c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0)) {
-    if (!ok(ptenc_launch_step_e1(c, l0, nl, true, sb + h.k, sb + h.v, act, nullptr, nullptr, nullptr, 0, st),
-            "decode_step_host/append_evict+encode", st))
-      return PTENC_ECUDA;
-  } else {
-    if (!ok(ptenc_launch_append_evict(c, l0, nl, sb + h.k, sb + h.v, act, nullptr, nullptr, nullptr, st),
-            "decode_step_host/append_evict", st))
-      return PTENC_ECUDA;
-    if (c->cfg.encode_enabled &&
-        !ok(ptenc_launch_encode(c, l0, nl, nullptr, nullptr, nullptr, 0, st), "decode_step_host/encode", st))
-      return PTENC_ECUDA;
-  }
+  if (!launch_append_and_encode(c, l0, nl, sb + h.k, sb + h.v, act, st, "decode_step_host")) return PTENC_ECUDA;
   // a2 group by group
   for (int g = 0; g < ng; ++g) {
     const int a0 = gb[g], a1 = gb[g + 1];
@@ -488,6 +529,30 @@ int ptenc_get_state(ptenc_cache* c, int layer, float* S_out, void* stream) {
   const size_t n = (size_t)d.B * d.G * d.r;
   return cudaMemcpyAsync(S_out, d.S + layer * n, n * 4, cudaMemcpyDeviceToDevice,
                          static_cast<cudaStream_t>(stream)) == cudaSuccess ? PTENC_OK : PTENC_ECUDA;
+}
+
+int ptenc_get_evicted(ptenc_cache* c, int layer, int64_t* tokens, int32_t* slots, int32_t* n_evicted, void* stream) {
+  if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers) return PTENC_EINVAL;
+  if (c->cfg.policy != PTENC_POLICY_SCORE) return PTENC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t B = c->cfg.batch, E = c->cfg.evict_chunk;
+  const PtencDev& d = c->dev;
+  if (tokens && cudaMemcpyAsync(tokens, d.ev_tok + layer * B * E, B * E * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (slots && cudaMemcpyAsync(slots, d.ev_slot + layer * B * E, B * E * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  if (n_evicted &&
+      cudaMemcpyAsync(n_evicted, d.n_staged + layer * B, B * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return PTENC_ECUDA;
+  return PTENC_OK;
+}
+
+int ptenc_get_scores(ptenc_cache* c, int layer, float* score_out, int32_t* token_out, void* stream) {
+  if (c == nullptr || layer < 0 || layer >= c->cfg.n_layers || score_out == nullptr || token_out == nullptr)
+    return PTENC_EINVAL;
+  if (c->cfg.policy != PTENC_POLICY_SCORE) return PTENC_EINVAL;
+  return ptenc_launch_export_scores(c, layer, score_out, token_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_cache_status(ptenc_cache* c, int32_t* dev_status) {

@@ -163,7 +163,10 @@ struct Smem {
 };
 
 // ------------------------------------------------------------------------------------------------ kernel
-template <int D, int TILE_N, int NW, int STAGES>
+// SCORE: the cache runs the importance-aware eviction policy.  Live slots are then given by a bitmap instead of a
+// ring interval, and the launch leaves behind what the policy needs to turn this attention into per-token mass: the
+// scaled logits of every live slot (base-2 domain, [unit][slot][8 heads]) and the log2-sum-exp2 of every query head.
+template <int D, int TILE_N, int NW, int STAGES, bool SCORE>
 __global__ void __launch_bounds__((NW + 1) * 32, PTENC_ATTN_CTAS_PER_SM)
 k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
@@ -211,9 +214,17 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     const int li = e / B, b = e - li * B;
     const size_t lb = (size_t)(l0 + li) * B + b;
     if (active != nullptr && active[b] == 0) return en;          // inactive: no tiles
-    en.head = p.head[lb];
-    en.count = p.count[lb];
     en.sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;
+    if (SCORE) {
+      // slots fill in order until the window is full and are reused in place afterwards: the slots in use are a
+      // prefix [0, min(n_appended, W)); which of them hold a token is the bitmap's business (see the mask below)
+      const long long n = p.n_app[lb];
+      en.head = 0;
+      en.count = (int)(n < (long long)W ? n : (long long)W) - en.sink;
+    } else {
+      en.head = p.head[lb];
+      en.count = p.count[lb];
+    }
     const int cap = W - en.sink;
     if (en.sink < 0 || cap < 1 || en.head < 0 || en.head >= cap || en.count < 0 || en.count > cap) {
       // a ring state outside its range (corrupt workspace, or bad head/count arrays handed to the static-scratch
@@ -394,6 +405,12 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       const uint32_t s = seq % STAGES;
       const int iu = (int)(lo - ub) + i;
       const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
+      uint32_t lw0 = 0xffffffffu, lw1 = 0xffffffffu;        // liveness of the tile's slots (SCORE), requested early
+      if (SCORE) {
+        const unsigned int* lw = p.live_bits + ((size_t)(l0 + li) * B + b) * p.wb + ((j * TILE_N) >> 5);
+        lw0 = lw[0];
+        if (TILE_N > 32) lw1 = lw[1];
+      }
       if (misc[0] == 0 && !mbar_wait(bar_full + 8 * s, (seq / STAGES) & 1)) {
         atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
         misc[0] = 1;
@@ -420,24 +437,49 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       }
       // ---- mask slots that hold no live token (rows qr and qr + 8 of each row tile) -------------------------------
       const int slot0 = j * TILE_N;
-      bool full = false;
-      if (slot0 + TILE_N <= sink) {
-        full = true;
-      } else if (slot0 >= sink && slot0 + TILE_N <= W) {
-        int d0 = slot0 - sink - head;
-        if (d0 < 0) d0 += cap;
-        full = (count == cap) || (d0 + TILE_N <= count);
-      }
-      if (!full) {
+      if (SCORE) {
+        if ((lw0 & lw1) != 0xffffffffu) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const int o = 16 * mt + qr + 8 * x;               // slot within the tile
+              const bool live = (((o < 32 ? lw0 : lw1) >> (o & 31)) & 1u) != 0;
+              if (!live) { sT[mt][2 * x] = -INFINITY; sT[mt][2 * x + 1] = -INFINITY; }
+            }
+          }
+        }
+        // scaled logits of the live slots: a lane holds heads 2 qc, 2 qc + 1 of tokens qr and qr + 8 of each row tile
+        float* lg = p.logits + ((((size_t)(l0 + li) * B + b) * Hkv + h) * W + slot0) * 8 + 2 * qc;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
           for (int x = 0; x < 2; ++x) {
-            const int slot = slot0 + 16 * mt + qr + 8 * x;
-            int dd = slot - sink - head;
-            if (dd < 0) dd += cap;
-            const bool live = slot < sink || (slot < W && dd < count);
-            if (!live) { sT[mt][2 * x] = -INFINITY; sT[mt][2 * x + 1] = -INFINITY; }
+            const int o = 16 * mt + qr + 8 * x;
+            if (sT[mt][2 * x] != -INFINITY && slot0 + o < W)
+              *reinterpret_cast<float2*>(lg + (size_t)o * 8) = make_float2(sT[mt][2 * x] * sl2, sT[mt][2 * x + 1] * sl2);
+          }
+        }
+      } else {
+        bool full = false;
+        if (slot0 + TILE_N <= sink) {
+          full = true;
+        } else if (slot0 >= sink && slot0 + TILE_N <= W) {
+          int d0 = slot0 - sink - head;
+          if (d0 < 0) d0 += cap;
+          full = (count == cap) || (d0 + TILE_N <= count);
+        }
+        if (!full) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const int slot = slot0 + 16 * mt + qr + 8 * x;
+              int dd = slot - sink - head;
+              if (dd < 0) dd += cap;
+              const bool live = slot < sink || (slot < W && dd < count);
+              if (!live) { sT[mt][2 * x] = -INFINITY; sT[mt][2 * x + 1] = -INFINITY; }
+            }
           }
         }
       }
@@ -560,7 +602,9 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
             out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
           }
           if (lse != nullptr && d0 == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
+          if (SCORE && d0 == 0) p.lse2[((size_t)(l0 + li) * B + b) * p.Hq + (size_t)h * g + r] = mt + log2f(lt);
         }
+        if (SCORE && tid == 0) p.pending[(size_t)(l0 + li) * B + b] = 1;
       } else {
 #pragma unroll
         for (int d = d0; d < D; d += TPR) {
@@ -607,7 +651,9 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
           }
           out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
           if (lse != nullptr && d == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
+          if (SCORE && d == 0) p.lse2[((size_t)(l0 + li) * B + b) * p.Hq + (size_t)h * g + r] = mt + log2f(lt);
         }
+        if (SCORE && tid == 0) p.pending[(size_t)(l0 + li) * B + b] = 1;
       }
     }
     consumer_sync(NCONS);       // merge buffers and misc[1] are free again
@@ -677,24 +723,34 @@ inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
   return n_t >= PTENC_ATTN_LONG_MIN_TILES_PER_UNIT && tiles >= PTENC_ATTN_LONG_MIN_TILES;
 }
 
-template <int D, int NW>
-cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
-                     cudaStream_t st) {
+template <int D, int NW, bool SCORE>
+cudaError_t launch_ts(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
+                      cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   const size_t smem = SM::TOTAL + 1024;
-  k_attn_bf16<D, TN, NW, STAGES><<<c->attn_grid, (NW + 1) * 32, smem, st>>>(
+  k_attn_bf16<D, TN, NW, STAGES, SCORE><<<c->attn_grid, (NW + 1) * 32, smem, st>>>(
       c->dev, c->tmK, c->tmV, l0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
   c->launches++;
   return cudaGetLastError();
+}
+template <int D, int NW>
+cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
+                     cudaStream_t st) {
+  return c->cfg.policy == PTENC_POLICY_SCORE ? launch_ts<D, NW, true>(c, l0, nl, q, active, out, lse, st)
+                                             : launch_ts<D, NW, false>(c, l0, nl, q, active, out, lse, st);
 }
 
 template <int D, int NW>
 cudaError_t prepare_nw() {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
-  return cudaFuncSetAttribute(k_attn_bf16<D, TN, NW, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              SM::TOTAL + 1024);
+  cudaError_t e = cudaFuncSetAttribute(k_attn_bf16<D, TN, NW, STAGES, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL + 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_attn_bf16<D, TN, NW, STAGES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SM::TOTAL + 1024);
+  return e;
 }
 template <int D>
 cudaError_t prepare_t() {
@@ -802,7 +858,7 @@ cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const C
                             const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
-  k_attn_bf16<D, TN, NW, STAGES><<<grid, (NW + 1) * 32, SM::TOTAL + 1024, st>>>(
+  k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 1) * 32, SM::TOTAL + 1024, st>>>(
       dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
   return cudaGetLastError();
 }

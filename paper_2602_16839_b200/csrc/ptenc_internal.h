@@ -41,6 +41,20 @@ struct PtencDev {
   int* tickets;                 // [L][B][Hkv] arrival counters, self-cleaning
   int part_slots;
   int* status;
+  // ---- importance-aware eviction (policy PTENC_POLICY_SCORE); all null / zero under the sliding-window policy -------
+  int policy, recent;
+  int wb;                       // 32-bit words of one sequence's liveness bitmap
+  int* slot_tok;                // [L][B][W] token index held by a slot (meaningful where the slot is live)
+  float* score;                 // [L][B][W] attention mass the slot's token has received so far
+  unsigned int* live_bits;      // [L][B][wb] bit s set = slot s holds a token (pinned entries included)
+  float* logits;                // [L][B][Hkv][W][8] scaled logits (base-2 domain) of the latest attention
+  float* lse2;                  // [L][B][Hq] log2-sum-exp2 of the latest attention
+  int* pending;                 // [L][B] 1 = the latest attention's mass has not been folded into the scores yet
+  int* fq;                      // [L][B][E] freed slots in the order they were freed
+  int* fq_head;                 // [L][B] next entry of fq to reuse
+  int* fq_count;                // [L][B] entries of fq not reused yet
+  long long* ev_tok;            // [L][B][E] tokens evicted by the last append, oldest first
+  int* ev_slot;                 // [L][B][E] their slots
 };
 
 struct ptenc_cache {
@@ -73,6 +87,14 @@ cudaError_t ptenc_launch_append_evict(ptenc_cache* c, int l0, int nl, const void
                                       const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
                                       int32_t* n_evicted_out, cudaStream_t st);
 cudaError_t ptenc_launch_reset(ptenc_cache* c, const uint8_t* seq_mask, cudaStream_t st);
+// Importance-aware policy: fold the latest attention's mass into the scores, evict the lowest-scoring candidates
+// when the cache is full (rows staged oldest first), store the arriving token in a freed slot.
+cudaError_t ptenc_launch_score_step(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
+                                    const uint8_t* active, int32_t* slot_out, int64_t* evict_first_out,
+                                    int32_t* n_evicted_out, cudaStream_t st);
+cudaError_t ptenc_launch_export_scores(ptenc_cache* c, int layer, float* score_out, int32_t* token_out,
+                                       cudaStream_t st);
+size_t ptenc_score_step_smem(const ptenc_config* cfg);
 cudaError_t ptenc_launch_prefill(ptenc_cache* c, int l0, int nl, const void* K_p, const void* V_p,
                                  const int32_t* n_prompt, int p_max, cudaStream_t st);
 cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,

@@ -108,7 +108,10 @@ __global__ void k_reset(PtencDev p, const uint8_t* __restrict__ mask, int clear_
     p.n_sink[lb] = 0;
     p.n_staged[lb] = 0;
     p.evict_first[lb] = -1;
+    if (p.policy == PTENC_POLICY_SCORE) { p.pending[lb] = 0; p.fq_head[lb] = 0; p.fq_count[lb] = 0; }
   }
+  if (p.policy == PTENC_POLICY_SCORE)                      // no slot holds a token any more
+    for (int i = threadIdx.x; i < p.wb; i += blockDim.x) p.live_bits[lb * p.wb + i] = 0u;
   const int gr = p.G * p.r;
   for (int i = threadIdx.x; i < gr; i += blockDim.x) p.S[lb * gr + i] = p.S0[(long long)l * gr + i];
 }
@@ -140,6 +143,14 @@ k_prefill(PtencDev p, int l0, const char* __restrict__ K_p, const char* __restri
     const size_t dst = (((size_t)lb * Hkv + h) * W + i) * rb + (size_t)v * 16;
     *reinterpret_cast<uint4*>(p.K + dst) = *reinterpret_cast<const uint4*>(K_p + src);
     *reinterpret_cast<uint4*>(p.V + dst) = *reinterpret_cast<const uint4*>(V_p + src);
+  }
+  if (p.policy == PTENC_POLICY_SCORE) {
+    // importance-aware policy: the pinned slots are live like any other; they are never candidates for eviction
+    for (int i = threadIdx.x; i < n; i += blockDim.x) { p.slot_tok[lb * W + i] = i; p.score[lb * W + i] = 0.f; }
+    for (int w = threadIdx.x; w < p.wb; w += blockDim.x) {
+      const int lo = w * 32;
+      p.live_bits[lb * p.wb + w] = n >= lo + 32 ? 0xffffffffu : (n > lo ? (1u << (n - lo)) - 1u : 0u);
+    }
   }
   __syncthreads();          // every thread has read n_app / count / n_sink above before they change
   if (threadIdx.x == 0) {

@@ -138,7 +138,7 @@ def test_needle_in_every_tile_small_shapes(warps, W, B):
     exactly full, and wrapped at an odd slot; most units split between CTAs (few units, 148 CTAs)."""
     c = {**CONFIGS["qwen7b"], "window": W, "batch": B}
     info, n = _run_needles(c, 2, [W - W // 3, W, W + W // 2 + 13], warps)
-    assert info["consumer_warps"] == warps and n >= 3 * 3 * 5
+    assert info["consumer_warps"] == warps and n >= 5 * sum((min(T, W) + 31) // 32 for T in (W - W // 3, W, W + 1))
 
 
 @pytest.mark.parametrize("name", ["qwen7b", "llama8b"])
