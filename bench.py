@@ -36,7 +36,8 @@ def _oracle_worker(path: str) -> None:
     n_seq, W, E, n_prompt = int(d["n_seq"]), int(d["window"]), int(d["evict_chunk"]), int(d["n_prompt"])
     orc = OracleCache(n_layers=1, batch=n_seq, n_q_heads=int(d["n_q_heads"]), n_kv_heads=int(d["n_kv_heads"]),
                       head_dim=int(d["head_dim"]), window=W, evict_chunk=E, n_global=int(d["n_global"]),
-                      rank=int(d["rank"]))
+                      rank=int(d["rank"]), policy="score" if int(d["score_policy"]) else "fifo",
+                      recent=int(d["recent"]) if int(d["score_policy"]) else 0)
     orc.set_encoder(0, **{k: d["enc_" + k] for k in ("Wq_a", "Wk_a", "Wv_a", "q_g", "k_g", "v_g")})
     q, k, v = d["q"], d["k"], d["v"]                      # [R, n_seq, H, D] each
     R = q.shape[0]
@@ -106,7 +107,7 @@ def evicts_at(t: int, W: int, E: int, P: int = 0) -> bool:
     return t >= cap and (t - cap) % min(E, cap) == 0
 
 
-def bytes_model(c: dict, E: int = 1, steps=None, P: int = 0) -> dict:
+def bytes_model(c: dict, E: int = 1, steps=None, P: int = 0, score_policy: bool = False) -> dict:
     """Algorithmic bytes (all layers, all sequences active) summed over the given steps (token indices); one
     full-window evicting step when `steps` is None.  Per layer and sequence: the live K and V rows + q + o for the
     attention, the arriving K/V rows for the append, and on an evicting step the E evicted K/V rows + the state read
@@ -124,6 +125,11 @@ def bytes_model(c: dict, E: int = 1, steps=None, P: int = 0) -> dict:
     attn = sum(L * B * (2 * n * d_kv * elt + 2 * d_q * elt) for n in live)          # K,V window + q + o
     append = len(live) * L * B * 2 * d_kv * elt
     enc = sum(L * B * (2 * min(E, W - P) * d_kv * elt + 2 * c["n_global"] * c["rank"] * 4) for e in ev if e)
+    if score_policy:
+        # importance-aware eviction: the per-slot scores are read and written once per step (fp32).  The logits that
+        # carry the attention mass from the attention kernel to the scores are this implementation's traffic, not the
+        # method's, and count against the achieved figure.
+        append += sum(L * B * 2 * (n - P) * 4 for n in live)
     return {"attn": attn, "step": attn + append + enc, "attn_per_step": [L * B * (2 * n * d_kv * elt + 2 * d_q * elt)
                                                                           for n in live]}
 
@@ -193,7 +199,8 @@ def host_cores() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, n_prompt: int = 0, workers: int = 1):
+def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, n_prompt: int = 0, workers: int = 1,
+                  policy: str = "fifo", recent: int = 0):
     """Times the CPU oracle, as it stands, on `workers` processes at once, each holding 1 layer x n_seq sequences of
     its own at the full window (sequences are independent, so this is how the oracle uses many cores).  Every
     process runs single-threaded; all start their timed steps together.  Returns (seconds per sampled step = the
@@ -211,7 +218,7 @@ def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, 
         kv = [gen.step_kv(t) for t in range(R)]
         arrays = dict(n_seq=n_seq, window=c["window"], evict_chunk=E, n_prompt=n_prompt, n_q_heads=c["n_q_heads"],
                       n_kv_heads=c["n_kv_heads"], head_dim=c["head_dim"], n_global=c["n_global"], rank=c["rank"],
-                      warm=warm, n_steps=n_steps, q=q, k=np.stack([x[0][0].double().numpy() for x in kv]),
+                      warm=warm, n_steps=n_steps, score_policy=int(policy == "score"), recent=recent, q=q, k=np.stack([x[0][0].double().numpy() for x in kv]),
                       v=np.stack([x[1][0].double().numpy() for x in kv]),
                       **{"enc_" + k: v.double().numpy() for k, v in P.items()})
         if n_prompt > 0:
@@ -251,14 +258,16 @@ def oracle_sample(c: dict, n_seq: int, n_steps: int, warm: int = 1, E: int = 1, 
     return wall / n_steps, workers, sum(r["cpu"] for r in res) / wall
 
 
-def oracle_baseline(c: dict, n_steps: int, E: int, n_prompt: int, warm: int = 1) -> dict:
+def oracle_baseline(c: dict, n_steps: int, E: int, n_prompt: int, warm: int = 1, policy: str = "fifo",
+                    recent: int = 0) -> dict:
     """The oracle on one core and on all host cores; tokens/s normalised to all L layers."""
     L, B, W = c["n_layers"], c["batch"], c["window"]
     nproc = host_cores()
     n1 = min(8, B)
-    sec1, _, busy1 = oracle_sample(c, n1, n_steps, warm=warm, E=E, n_prompt=n_prompt, workers=1)
+    kw = dict(warm=warm, E=E, n_prompt=n_prompt, policy=policy, recent=recent)
+    sec1, _, busy1 = oracle_sample(c, n1, n_steps, workers=1, **kw)
     nw = 2                                                   # sequences per process on the all-cores leg
-    secN, P, busyN = oracle_sample(c, nw, n_steps, warm=warm, E=E, n_prompt=n_prompt, workers=nproc)
+    secN, P, busyN = oracle_sample(c, nw, n_steps, workers=nproc, **kw)
     return {
         "value": P * nw / (secN * L), "unit": UNIT, "cores": P, "nproc": nproc, "kind": "oracle",
         "cpu_seconds_per_wall_second": busyN,
@@ -276,7 +285,8 @@ def run_reference(args, c: dict):
     """--impl reference: the oracle on a bounded sample; tokens/s normalised to all L layers."""
     if rank_env()[0] != 0:
         return
-    base = oracle_baseline(c, max(1, args.steps), args.evict_chunk, args.prompt_len, warm=max(1, args.warmup))
+    base = oracle_baseline(c, max(1, args.steps), args.evict_chunk, args.prompt_len, warm=max(1, args.warmup),
+                           policy=args.policy, recent=args.recent)
     L, B = c["n_layers"], c["batch"]
     seqs = base["cores"] * 2
     line = {
@@ -306,7 +316,8 @@ def l2_note(c: dict) -> str:
 def config_block(args, c: dict) -> dict:
     return {"workload": args.workload, "n_layers": c["n_layers"], "batch_per_gpu": c["batch"],
             "n_q_heads": c["n_q_heads"], "n_kv_heads": c["n_kv_heads"], "head_dim": c["head_dim"],
-            "window": c["window"], "evict_chunk": args.evict_chunk, "pinned_prompt": args.prompt_len, "n_global": c["n_global"], "rank": c["rank"],
+            "window": c["window"], "evict_chunk": args.evict_chunk, "pinned_prompt": args.prompt_len,
+            "policy": args.policy + (f" (recent {args.recent})" if args.policy == "score" else ""), "n_global": c["n_global"], "rank": c["rank"],
             "phase": ("steady state: rings full, one eviction + encode per sequence per step" if args.evict_chunk == 1
                       else f"steady state: rings between {c['window'] - args.evict_chunk + 1} and {c['window']} tokens, "
                            f"every {args.evict_chunk}-th step evicts and encodes {args.evict_chunk} tokens per sequence"),
@@ -398,8 +409,11 @@ def run_gpu(args, c: dict):
     L, B, Hq, Hkv, D, W = c["n_layers"], c["batch"], c["n_q_heads"], c["n_kv_heads"], c["head_dim"], c["window"]
     gen = make_inputs(c, seed=shard_seed(rank), device=dev)
     E = args.evict_chunk
+    score_policy = args.policy == "score"
     cfg = pt.make_config(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, window=W, evict_chunk=E,
-                         n_global=c["n_global"], rank=c["rank"], dtype=c["dtype"], device=local)
+                         n_global=c["n_global"], rank=c["rank"], dtype=c["dtype"], device=local,
+                         policy=pt.binding.POLICY_SCORE if score_policy else pt.binding.POLICY_FIFO,
+                         recent=args.recent if score_policy else 0)
     cache = pt.Cache(cfg)
     for l in range(L):
         P = gen.encoder_params(l)
@@ -450,13 +464,23 @@ def run_gpu(args, c: dict):
     torch.cuda.nvtx.range_push("ptenc_timed")
     e0.record()
     for t in range(K):
-        cache.time_next_attn(ev_a[t], ev_b[t])
         cache.decode_step(-1, *pool[t % R], out)
     e1.record()
     sync_all()
-    torch.cuda.nvtx.range_pop()
     ms_total = e0.elapsed_time(e1)
     launches = cache.launch_count() - launches0
+    # the same K steps once more with an event pair around every attention launch (for the roofline of that kernel);
+    # an event in front of the launch makes it an ordinary serialised launch, so these steps are a little slower than
+    # the ones timed above and are not part of `value`
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for t in range(K):
+        cache.time_next_attn(ev_a[t], ev_b[t])
+        cache.decode_step(-1, *pool[(K + t) % R], out)
+    e3.record()
+    sync_all()
+    torch.cuda.nvtx.range_pop()
+    ms_total_events = e2.elapsed_time(e3)
     attn_ms = [a.elapsed_time(b) for a, b in zip(ev_a, ev_b)]
     clocks = sampler.stop() if sampler else None
     status = cache.status()
@@ -499,7 +523,7 @@ def run_gpu(args, c: dict):
         if E > 1:
             # the encoder's burst: every sequence folds a chunk of E staged rows (the rows staged by the last evicting
             # step are folded again on each call; the arithmetic and the traffic are those of a real burst)
-            n_done = (W - P) + Wm + K + 3 + Ke                    # decoded tokens so far (fill, warm-up, both timed loops)
+            n_done = (W - P) + Wm + 2 * K + 3 + Ke                # decoded tokens so far (fill, warm-up, the timed loops)
             t = n_done
             while not evicts_at(t, W, E, P):
                 t += 1
@@ -529,11 +553,12 @@ def run_gpu(args, c: dict):
 
     if rank == 0:
         timed_tokens = list(range(W - P + Wm, W - P + Wm + K))  # decoded-token index arriving at each timed step
-        bm = bytes_model(c, E, timed_tokens, P)
+        bm = bytes_model(c, E, timed_tokens, P, score_policy)
+        bm_ev = bytes_model(c, E, [t + K for t in timed_tokens], P, score_policy)     # the pass with events
         peak, peak_kind = measured_peak()
         ms_step = ms_total / K
         attn_avg_ms = sum(attn_ms) / len(attn_ms)
-        attn_gbs = bm["attn"] / (sum(attn_ms) * 1e-3) / 1e9
+        attn_gbs = bm_ev["attn"] / (sum(attn_ms) * 1e-3) / 1e9
         step_gbs = bm["step"] / (ms_total * 1e-3) / 1e9
         bm["attn"] /= K                                          # per launch / per step averages from here on
         bm["step"] /= K
@@ -555,14 +580,16 @@ def run_gpu(args, c: dict):
                          "peak": peak, "peak_kind": f"of {peak_kind} copy bandwidth", "unit": "GB/s",
                          "frac": attn_gbs / peak, "frac_of_8tbs": attn_gbs / NOMINAL_HBM_GBS,
                          "traffic": traffic, "algorithmic_bytes_per_launch": bm["attn"],
-                         "avg_launch_ms": attn_avg_ms, "share_of_step": attn_avg_ms / ms_step},
+                         "avg_launch_ms": attn_avg_ms, "share_of_step": attn_avg_ms / (ms_total_events / K),
+                         "timed": f"{K} launches with an event pair each, in a second pass over the same steps "
+                                  f"({ms_total_events / K:.4f} ms per step with the events in place)"},
             "hbm": {"step_algorithmic_gbs": step_gbs, "frac_of_8tbs": step_gbs / NOMINAL_HBM_GBS,
                     "frac_of_measured": step_gbs / peak, "algorithmic_bytes_per_step": bm["step"]},
             "device_status": status,
             **({"extras": extras} if extras else {}),
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = oracle_baseline(c, args.cpu_steps, E, P)
+            line["cpu_baseline"] = oracle_baseline(c, args.cpu_steps, E, P, policy=args.policy, recent=args.recent)
         print(json.dumps(line), flush=True)
     cache.close()
     if dist is not None:
@@ -585,6 +612,11 @@ def main():
     ap.add_argument("--prompt-len", type=int, default=0,
                     help="tokens of a pinned prompt per sequence (kept for the whole rollout; the window slides over "
                          "the remaining slots)")
+    ap.add_argument("--policy", default="fifo", choices=["fifo", "score"],
+                    help="which tokens leave a full cache: the oldest (sliding window, the timed configuration) or the "
+                         "ones that received the least attention so far (Sec. 4.3, token dropping)")
+    ap.add_argument("--recent", type=int, default=256,
+                    help="--policy score: the newest RECENT tokens are never evicted")
     ap.add_argument("--cpu-steps", type=int, default=96, help="steps of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dry-run", action="store_true",

@@ -148,11 +148,11 @@ bool launch_append_and_encode(ptenc_cache* c, int l0, int nl, const void* k_new,
 }
 
 cudaError_t launch_attn(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
-                        float* lse, bool fold_staged, cudaStream_t st) {
+                        float* lse, bool fold_staged, bool early, cudaStream_t st) {
   cudaEvent_t e0 = c->ev_attn_begin, e1 = c->ev_attn_end;
   c->ev_attn_begin = c->ev_attn_end = nullptr;
-  if (e0 != nullptr) cudaEventRecord(e0, st);
-  cudaError_t rc = c->fast_attn ? ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, fold_staged, st)
+  if (e0 != nullptr) { cudaEventRecord(e0, st); early = false; }   // an event in between: an ordinary launch
+  cudaError_t rc = c->fast_attn ? ptenc_launch_attn_bf16(c, l0, nl, q, active, out, lse, fold_staged, early, st)
                                 : ptenc_launch_attn_generic(c, l0, nl, q, active, out, lse, st);
   if (e1 != nullptr) cudaEventRecord(e1, st);
   return rc;
@@ -350,7 +350,7 @@ int ptenc_decode_attn(ptenc_cache* c, int layer, const void* q, const uint8_t* a
   if (q == nullptr || out == nullptr) return PTENC_EINVAL;
   if (misaligned(q) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return ok(launch_attn(c, l0, nl, q, active, out, lse_out, false, st), "decode_attn", st) ? PTENC_OK : PTENC_ECUDA;
+  return ok(launch_attn(c, l0, nl, q, active, out, lse_out, false, false, st), "decode_attn", st) ? PTENC_OK : PTENC_ECUDA;
 }
 
 int ptenc_encode(ptenc_cache* c, int layer, const void* K_e, const void* V_e, const int32_t* n_evicted,
@@ -390,7 +390,8 @@ int ptenc_decode_step(ptenc_cache* c, int layer, const void* q, const void* k_ne
   if (misaligned(q) || misaligned(k_new) || misaligned(v_new) || misaligned(out)) return PTENC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!launch_append_and_encode(c, l0, nl, k_new, v_new, active, st)) return PTENC_ECUDA;
-  if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, step_folds_in_attention(c), st), "decode_step/attn", st))
+  const bool fold = step_folds_in_attention(c);
+  if (!ok(launch_attn(c, l0, nl, q, active, out, nullptr, fold, fold && !debug_on(), st), "decode_step/attn", st))
     return PTENC_ECUDA;
   return PTENC_OK;
 }
@@ -500,7 +501,7 @@ int ptenc_decode_step_host(ptenc_cache* c, int layer, const void* q_host, const 
     const int a0 = gb[g], a1 = gb[g + 1];
     if (!good(cudaStreamWaitEvent(st, c->ev_q[g], 0))) return PTENC_ECUDA;
     if (!ok(launch_attn(c, l0 + a0, a1 - a0, sb + h.q + a0 * q_layer, act, sb + h.out + a0 * q_layer, nullptr,
-                        step_folds_in_attention(c), st),
+                        step_folds_in_attention(c), false, st),
             "decode_step_host/attn", st))
       return PTENC_ECUDA;
     if (!good(cudaEventRecord(c->ev_o[g], st)) || !good(cudaStreamWaitEvent(c->st_out, c->ev_o[g], 0)) ||

@@ -23,8 +23,8 @@
 //    No CTA ever waits for another.
 //  * Every mbarrier wait is bounded; when one runs out the CTA raises a status bit, stops waiting and runs
 //    to completion on whatever is in shared memory, so barriers stay matched and nothing hangs.
-//  * One more warp per CTA is the step's encoder (Sec. 3.3, Eq. (3)): in a fused ring-per-step decode step it folds
-//    the rows that the append of the same step evicted into the states, a (layer, sequence) at a time, while the
+//  * Two more warps per CTA are the step's encoders (Sec. 3.3, Eq. (3)): in a fused ring-per-step decode step it folds
+//    the rows that the append of the same step evicted into the states, a (layer, sequence) at a time each, while the
 //    other warps stream K/V.  The attention of a step does not read the state, so the two are independent; the
 //    encoder's traffic (one evicted row, the encoder weights from L2, 8 KiB of state) is noise beside the K/V stream,
 //    and its chain of dependent memory round trips no longer sits in front of the attention.
@@ -46,6 +46,9 @@
 #endif
 #ifndef PTENC_ATTN_CTAS_PER_SM
 #define PTENC_ATTN_CTAS_PER_SM 1
+#endif
+#ifndef PTENC_ATTN_ENC_WARPS
+#define PTENC_ATTN_ENC_WARPS 2          // warps that fold staged rows while the others stream K/V
 #endif
 #ifndef PTENC_ATTN_L2PROMO
 #define PTENC_ATTN_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
@@ -173,12 +176,13 @@ struct Smem {
 // ring interval, and the launch leaves behind what the policy needs to turn this attention into per-token mass: the
 // scaled logits of every live slot (base-2 domain, [unit][slot][8 heads]) and the log2-sum-exp2 of every query head.
 template <int D, int TILE_N, int NW, int STAGES, bool SCORE>
-__global__ void __launch_bounds__((NW + 2) * 32, PTENC_ATTN_CTAS_PER_SM)
+__global__ void __launch_bounds__((NW + 1 + PTENC_ATTN_ENC_WARPS) * 32, PTENC_ATTN_CTAS_PER_SM)
 k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
             __nv_bfloat16* __restrict__ out, float* __restrict__ lse, const int fold_staged) {
   using SM = Smem<D, TILE_N, NW, STAGES>;
-  constexpr int NTHREADS = (NW + 2) * 32;                    // consumers, the TMA producer, the encoder
+  constexpr int NE = PTENC_ATTN_ENC_WARPS;
+  constexpr int NTHREADS = (NW + 1 + NE) * 32;               // consumers, the TMA producer, the encoder warps
   constexpr int NCONS = NW * 32;
   constexpr int KSTEPS = D / 16;
   constexpr int HALF_BYTES = TILE_N * 128;     // one 64-column half of a tile
@@ -211,6 +215,10 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   }
   for (int i = tid; i < 2 * SM::Q_BYTES / 4; i += NTHREADS) reinterpret_cast<uint32_t*>(smem + SM::OFF_Q)[i] = 0u;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  // When the launch was allowed to start before the kernel in front of it on the stream has finished (the fused
+  // step does that with its append/evict kernel), everything up to here overlapped that kernel; nothing it wrote is
+  // read before this point.  A no-op for an ordinary launch.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // ---- schedule: total tile count and this CTA's starting entry ------------------------------------
   struct Raw { int head, count, sink, act; long long n; };
@@ -293,11 +301,13 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   }
   __syncthreads();
 
-  if (warp == NW + 1) {
-    // ================================================================ encoder warp (see the file header)
-    // (layer, sequence) pairs of the call, dealt round-robin to the CTAs; it takes no part in anything below
+  if (warp > NW) {
+    // ================================================================ encoder warps (see the file header)
+    // (layer, sequence) pairs of the call, dealt round-robin to the encoder warps of all CTAs; they take no part in
+    // anything below.  Under the K/V stream a dependent memory round trip takes microseconds, and a pair is a chain
+    // of about a dozen: several warps per CTA keep the chain off the critical path at any batch size.
     if (fold_staged && p.encode_enabled) {
-      for (int e = blockIdx.x; e < n_ent; e += gridDim.x) {
+      for (int e = blockIdx.x * NE + (warp - NW - 1); e < n_ent; e += gridDim.x * NE) {
         const int li = e / B, b = e - li * B;
         const int l = l0 + li;
         const size_t lb = (size_t)l * B + b;
@@ -768,20 +778,35 @@ inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
 
 template <int D, int NW, bool SCORE>
 cudaError_t launch_ts(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
-                      bool fold_staged, cudaStream_t st) {
+                      bool fold_staged, bool early, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
-  const size_t smem = SM::TOTAL + 1024;
-  k_attn_bf16<D, TN, NW, STAGES, SCORE><<<c->attn_grid, (NW + 2) * 32, smem, st>>>(
-      c->dev, c->tmK, c->tmV, l0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, fold_staged ? 1 : 0);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(c->attn_grid);
+  cfg.blockDim = dim3((NW + 1 + PTENC_ATTN_ENC_WARPS) * 32);
+  cfg.dynamicSmemBytes = SM::TOTAL + 1024;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (early) {
+    // programmatic dependent launch: the grid may become resident and run its set-up while the kernel in front of it
+    // on the stream (which signals that it allows this) is still running; the kernel waits before its first read
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_attn_bf16<D, TN, NW, STAGES, SCORE>, c->dev, c->tmK, c->tmV, l0, nl,
+                                     (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, fold_staged ? 1 : 0);
   c->launches++;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 template <int D, int NW>
 cudaError_t launch_t(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
-                     bool fold_staged, cudaStream_t st) {
-  return c->cfg.policy == PTENC_POLICY_SCORE ? launch_ts<D, NW, true>(c, l0, nl, q, active, out, lse, fold_staged, st)
-                                             : launch_ts<D, NW, false>(c, l0, nl, q, active, out, lse, fold_staged, st);
+                     bool fold_staged, bool early, cudaStream_t st) {
+  return c->cfg.policy == PTENC_POLICY_SCORE
+             ? launch_ts<D, NW, true>(c, l0, nl, q, active, out, lse, fold_staged, early, st)
+             : launch_ts<D, NW, false>(c, l0, nl, q, active, out, lse, fold_staged, early, st);
 }
 
 template <int D, int NW>
@@ -830,13 +855,13 @@ void ptenc_attn_bf16_plan(const ptenc_cache* c, int nl, int* consumer_warps, int
 }
 
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out,
-                                   float* lse, bool fold_staged, cudaStream_t st) {
+                                   float* lse, bool fold_staged, bool early, cudaStream_t st) {
   const bool d128 = c->cfg.head_dim == 128;
   const bool lng = use_long_variant(c->cfg, nl, d128 ? Pick<128>::TILE_N : Pick<64>::TILE_N);
-  if (d128) return lng ? launch_t<128, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, st)
-                       : launch_t<128, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, st);
-  return lng ? launch_t<64, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, st)
-             : launch_t<64, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, st);
+  if (d128) return lng ? launch_t<128, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, early, st)
+                       : launch_t<128, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, early, st);
+  return lng ? launch_t<64, NW_LONG>(c, l0, nl, q, active, out, lse, fold_staged, early, st)
+             : launch_t<64, NW_DEFAULT>(c, l0, nl, q, active, out, lse, fold_staged, early, st);
 }
 
 // ================================================================================================================
@@ -901,7 +926,7 @@ cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const C
                             const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
-  k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 2) * 32, SM::TOTAL + 1024, st>>>(
+  k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 1 + PTENC_ATTN_ENC_WARPS) * 32, SM::TOTAL + 1024, st>>>(
       dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, 0);
   return cudaGetLastError();
 }

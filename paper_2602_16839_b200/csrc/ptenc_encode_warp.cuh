@@ -14,6 +14,7 @@
 
 constexpr int ENCW_MAX_VEC = 4;        // 16-byte vectors of a row held per lane: d_kv <= 32 * 4 * 8 = 1024
 constexpr int ENCW_MAX_RB = 4;         // 32-wide blocks of the rank: r <= 128
+constexpr int ENCW_JB = 4;             // output rows whose weights are in flight together
 
 __device__ __forceinline__ float encw_dot8(const uint4& w, const uint4& x) {
   const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&w);
@@ -53,41 +54,51 @@ __device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t l
   const __nv_bfloat16* Wv = reinterpret_cast<const __nv_bfloat16*>(p.Wv) + (size_t)l * r * d_kv;
 
   // ---- k_a = W^a_K k_e, v_a = W^a_V v_e: element j ends up in lane j % 32, register j / 32 ------------------------------
+  // The weights come from L2; a batch of ENCW_JB output rows is requested before any of it is used, so that a batch
+  // costs one round trip, not one per row.
   float ka[ENCW_MAX_RB], va[ENCW_MAX_RB];
 #pragma unroll
-  for (int jb = 0; jb < ENCW_MAX_RB; ++jb) {
-    ka[jb] = 0.f;
-    va[jb] = 0.f;
-    if (jb * 32 < r) {
-#pragma unroll 4
-      for (int jj = 0; jj < 32; ++jj) {
-        const int j = jb * 32 + jj;
-        if (j < r) {                                         // uniform over the warp
-          float sk = 0.f, sv = 0.f;
+  for (int jb = 0; jb < ENCW_MAX_RB; ++jb) { ka[jb] = 0.f; va[jb] = 0.f; }
+  for (int j0 = 0; j0 < r; j0 += ENCW_JB) {                  // r is a multiple of 8
+    uint4 wk[ENCW_JB][ENCW_MAX_VEC], wv[ENCW_JB][ENCW_MAX_VEC];
 #pragma unroll
-          for (int u = 0; u < ENCW_MAX_VEC; ++u) {
-            const int v = lane + 32 * u;
-            if (v < nv) {
-              const uint4 wk = __ldg(reinterpret_cast<const uint4*>(Wk + (size_t)j * d_kv + (size_t)v * 8));
-              const uint4 wv = __ldg(reinterpret_cast<const uint4*>(Wv + (size_t)j * d_kv + (size_t)v * 8));
-              sk += encw_dot8(wk, xk[u]);
-              sv += encw_dot8(wv, xv[u]);
-            }
-          }
+    for (int jj = 0; jj < ENCW_JB; ++jj) {
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            sk += __shfl_xor_sync(0xffffffffu, sk, o);
-            sv += __shfl_xor_sync(0xffffffffu, sv, o);
-          }
-          if (lane == jj) { ka[jb] = sk; va[jb] = sv; }
+      for (int u = 0; u < ENCW_MAX_VEC; ++u) {
+        const int v = lane + 32 * u;
+        if (v < nv) {
+          wk[jj][u] = __ldg(reinterpret_cast<const uint4*>(Wk + (size_t)(j0 + jj) * d_kv + (size_t)v * 8));
+          wv[jj][u] = __ldg(reinterpret_cast<const uint4*>(Wv + (size_t)(j0 + jj) * d_kv + (size_t)v * 8));
         }
       }
+    }
+#pragma unroll
+    for (int jj = 0; jj < ENCW_JB; ++jj) {
+      float sk = 0.f, sv = 0.f;
+#pragma unroll
+      for (int u = 0; u < ENCW_MAX_VEC; ++u) {
+        if (lane + 32 * u < nv) {
+          sk += encw_dot8(wk[jj][u], xk[u]);
+          sv += encw_dot8(wv[jj][u], xv[u]);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        sk += __shfl_xor_sync(0xffffffffu, sk, o);
+        sv += __shfl_xor_sync(0xffffffffu, sv, o);
+      }
+      const int j = j0 + jj;
+#pragma unroll
+      for (int jb = 0; jb < ENCW_MAX_RB; ++jb)
+        if ((j >> 5) == jb && lane == (j & 31)) { ka[jb] = sk; va[jb] = sv; }
     }
   }
 
   // ---- p = Q_a k_a; S <- Normalize(S + p v_a^T): a state row per lane -----------------------------------------------------
+  // Rows are moved 32 values (eight 16-byte loads in flight) at a time.
   const float* Qa = p.Qa + (size_t)l * G * r;
   float* S = p.S + lb * (size_t)G * r;
+  const bool row_mode = p.norm_mode == PTENC_NORM_ROW_L2;
   float total = 0.f;
   for (int g0 = 0; g0 < G; g0 += 32) {
     const int g = g0 + lane;
@@ -98,36 +109,53 @@ __device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t l
 #pragma unroll
     for (int jb = 0; jb < ENCW_MAX_RB; ++jb) {
       if (jb * 32 < r) {
-        for (int jj = 0; jj < 32 && jb * 32 + jj < r; jj += 4) {
-          const float4 qv = *reinterpret_cast<const float4*>(qrow + jb * 32 + jj);
-          pg = fmaf(qv.x, __shfl_sync(0xffffffffu, ka[jb], jj), pg);
-          pg = fmaf(qv.y, __shfl_sync(0xffffffffu, ka[jb], jj + 1), pg);
-          pg = fmaf(qv.z, __shfl_sync(0xffffffffu, ka[jb], jj + 2), pg);
-          pg = fmaf(qv.w, __shfl_sync(0xffffffffu, ka[jb], jj + 3), pg);
+        float4 qv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          qv[i] = (jb * 32 + 4 * i < r) ? *reinterpret_cast<const float4*>(qrow + jb * 32 + 4 * i)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {                        // lanes past r hold zeros in ka
+          pg = fmaf(qv[i].x, __shfl_sync(0xffffffffu, ka[jb], 4 * i), pg);
+          pg = fmaf(qv[i].y, __shfl_sync(0xffffffffu, ka[jb], 4 * i + 1), pg);
+          pg = fmaf(qv[i].z, __shfl_sync(0xffffffffu, ka[jb], 4 * i + 2), pg);
+          pg = fmaf(qv[i].w, __shfl_sync(0xffffffffu, ka[jb], 4 * i + 3), pg);
         }
       }
     }
     float ss = 0.f;
+    const bool one_block = r <= 32;                          // the whole row fits the registers: scale before storing
 #pragma unroll
     for (int jb = 0; jb < ENCW_MAX_RB; ++jb) {
       if (jb * 32 < r) {
-        for (int jj = 0; jj < 32 && jb * 32 + jj < r; jj += 4) {
-          float4 sv = *reinterpret_cast<const float4*>(srow + jb * 32 + jj);
-          sv.x = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], jj), sv.x);
-          sv.y = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], jj + 1), sv.y);
-          sv.z = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], jj + 2), sv.z);
-          sv.w = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], jj + 3), sv.w);
-          ss = fmaf(sv.x, sv.x, ss);
-          ss = fmaf(sv.y, sv.y, ss);
-          ss = fmaf(sv.z, sv.z, ss);
-          ss = fmaf(sv.w, sv.w, ss);
-          if (valid) *reinterpret_cast<float4*>(srow + jb * 32 + jj) = sv;       // the un-normalised sum
+        float4 sv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          sv[i] = (jb * 32 + 4 * i < r) ? *reinterpret_cast<const float4*>(srow + jb * 32 + 4 * i)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          sv[i].x = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], 4 * i), sv[i].x);
+          sv[i].y = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], 4 * i + 1), sv[i].y);
+          sv[i].z = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], 4 * i + 2), sv[i].z);
+          sv[i].w = fmaf(pg, __shfl_sync(0xffffffffu, va[jb], 4 * i + 3), sv[i].w);
+          ss = fmaf(sv[i].x, sv[i].x, ss);
+          ss = fmaf(sv[i].y, sv[i].y, ss);
+          ss = fmaf(sv[i].z, sv[i].z, ss);
+          ss = fmaf(sv[i].w, sv[i].w, ss);
+        }
+        const float sc = (one_block && row_mode) ? rsqrtf(fmaxf(ss, 1e-24f)) : 1.f;      // 1 / max(|row|, 1e-12)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (valid && jb * 32 + 4 * i < r)
+            *reinterpret_cast<float4*>(srow + jb * 32 + 4 * i) =
+                make_float4(sv[i].x * sc, sv[i].y * sc, sv[i].z * sc, sv[i].w * sc);
         }
       }
     }
     if (valid) total += ss;
-    if (p.norm_mode == PTENC_NORM_ROW_L2 && valid) {
-      const float sc = rsqrtf(fmaxf(ss, 1e-24f));            // 1 / max(|row|, 1e-12)
+    if (row_mode && !one_block && valid) {                   // longer rows were stored un-normalised: rescale them
+      const float sc = rsqrtf(fmaxf(ss, 1e-24f));
       for (int j = 0; j < r; j += 4) {
         float4 sv = *reinterpret_cast<const float4*>(srow + j);
         sv.x *= sc; sv.y *= sc; sv.z *= sc; sv.w *= sc;

@@ -105,8 +105,10 @@ cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void
                                       void* out, float* lse, cudaStream_t st);
 // fold_staged: the kernel's spare warp also folds the rows staged by the append of the same step (E = 1) into the
 // states of the layers of the call, while the K/V stream runs.
+// early: the launch directly follows ptenc_launch_ring_e1 on the same stream and may start while that kernel runs
+// (programmatic dependent launch); the attention kernel waits for it before its first read.
 cudaError_t ptenc_launch_attn_bf16(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
-                                   void* out, float* lse, bool fold_staged, cudaStream_t st);
+                                   void* out, float* lse, bool fold_staged, bool early, cudaStream_t st);
 // One evicted token per sequence (E = 1 on the staged path, or caller rows with m_max == 1), bf16, shapes the
 // one-warp encoder covers.  ring_e1: the append/evict alone (rows staged); encode_e1: the fold alone.
 bool ptenc_step_e1_usable(const ptenc_cache* c, const void* Ke, int m_max);

@@ -4,6 +4,8 @@
 // three thin products per sequence (r x d_in, G x r, d_out x G).  Each sequence has its own state, so this is a
 // batch of tiny products; the only sizeable traffic is A and B, which a CTA reads once for a block of sequences.
 // fp32 accumulation throughout; x, y, A, B in the storage dtype.
+#include <cooperative_groups.h>
+
 #include "ptenc_internal.h"
 
 namespace {
@@ -144,17 +146,23 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// bf16 path on warp-level mma.  Sixteen sequences are the 16 rows of the A operand.  Both thin products against the
-// weights run on the tensor cores so that the arithmetic and the bf16 unpacking leave the issue slots to the loads:
-//   u = X B^T   : A fragments straight from the inputs, B fragments straight from B (both L2), the column tiles of u
-//                 and splits of d_in spread over the 16 warps;
-//   y += w A^T  : w = S u is fp32; it is split into two bf16 terms w_hi + w_lo so that nothing but the final
-//                 rounding of y is lost, and A's rows are the B operand, again straight from L2.
-// A lane's 8 consecutive contraction values feed two mma steps; the contraction index is permuted the same way on
-// both operands, which leaves the sums unchanged.  S u in between is fp32 FMA, a warp per sequence.
+// bf16 path: warp-level mma inside a thread-block cluster.  Sixteen sequences are the 16 rows of the A operand; the
+// four CTAs of a cluster share one (layer, block of 16 sequences):
+//   phase 1  u = X B^T     each CTA contracts its quarter of d_in (A fragments straight from the inputs, B fragments
+//                          straight from B, both with one 16-byte load per lane feeding two mma steps; the contraction
+//                          index is permuted the same way on both operands, which leaves the sums unchanged); the
+//                          partial sums meet through distributed shared memory;
+//   phase 2  w = S u       fp32, each CTA for four of the sixteen sequences, a lane per state row; w is split into two
+//                          bf16 terms w_hi + w_lo so that nothing but the final rounding of y is lost; the quarters are
+//                          gathered through distributed shared memory;
+//   phase 3  y += w A^T    each CTA for its quarter of d_out, A's rows as the B operand.
+// Splitting a block four ways makes the call 4 x as many, smaller CTAs: all of them are resident at once (one wave),
+// every weight byte is still read once per 16 sequences, and the three dependent phases of one block overlap with
+// those of the others on the same SM.
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int LM_SEQ = 16;
-constexpr int LM_THREADS = 512;
+constexpr int LM_CLUSTER = 4;
+constexpr int LM_THREADS = 256;
 constexpr int LM_WARPS = LM_THREADS / 32;
 
 __device__ __forceinline__ void lr_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -173,27 +181,32 @@ __host__ __device__ inline int lm_k_split(int r) {
   return tiles < LM_WARPS ? LM_WARPS / tiles : 1;
 }
 __host__ __device__ inline size_t lr_mma_smem(int G, int r) {
-  // u [KS][16][r] fp32 | w_hi, w_lo [16][G] bf16
-  return (size_t)lm_k_split(r) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
+  // u partials [KS][16][r] fp32 | u of this CTA [16][r] fp32 | w_hi, w_lo [16][G] bf16
+  return (size_t)(lm_k_split(r) + 1) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
 }
 
-__global__ void __launch_bounds__(LM_THREADS)
-k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ Bm,
-                 const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
-                 const uint8_t* __restrict__ active, int d_in, int d_out) {
+// grid = (LM_CLUSTER, nl * ceil(B / 16)), cluster = (LM_CLUSTER, 1, 1)
+__global__ void __cluster_dims__(LM_CLUSTER, 1, 1) __launch_bounds__(LM_THREADS)
+k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ Bm,
+                     const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
+                     const uint8_t* __restrict__ active, int d_in, int d_out) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) uint8_t lm_smem[];
   const int G = p.G, r = p.r, B = p.B;
   const int n_tiles = r >> 3;                                   // column tiles of u
-  const int KS = lm_k_split(r);                                 // warps sharing a tile split d_in
-  float* u = reinterpret_cast<float*>(lm_smem);                 // [KS][16][r]
-  __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u + KS * LM_SEQ * r);   // [16][G]
+  const int KS = lm_k_split(r);                                 // warps sharing a tile split the CTA's slice of d_in
+  float* u_part = reinterpret_cast<float*>(lm_smem);            // [KS][16][r]
+  float* u_loc = u_part + KS * LM_SEQ * r;                      // [16][r] this CTA's share of the contraction
+  __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u_loc + LM_SEQ * r);    // [16][G]
   __nv_bfloat16* w_lo = w_hi + LM_SEQ * G;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qrow = lane >> 2, qcol = lane & 3;
+  const int rank = (int)cluster.block_rank();                   // = blockIdx.x
   const int nblk = (B + LM_SEQ - 1) / LM_SEQ;
-  const int li = blockIdx.x / nblk;
-  const int b0 = (blockIdx.x - li * nblk) * LM_SEQ;
+  const int li = blockIdx.y / nblk;
+  const int b0 = (blockIdx.y - li * nblk) * LM_SEQ;
   const int l = l0 + li;
   const int nseq = min(LM_SEQ, B - b0);
   const __nv_bfloat16* Bl = Bm + (size_t)li * r * d_in;
@@ -202,28 +215,36 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
   __nv_bfloat16* yl = y + ((size_t)li * B + b0) * d_out;
   const bool lo_ok = qrow < nseq, hi_ok = qrow + 8 < nseq;      // the two sequences whose rows this lane touches
 
+  // this CTA's shares: pairs of mma steps along d_in, tiles of 8 outputs along d_out, sequences of the block
+  const int n_pairs = d_in >> 5;
+  const int p_lo = rank * n_pairs / LM_CLUSTER, p_hi = (rank + 1) * n_pairs / LM_CLUSTER;
+  const int n_out_tiles = d_out >> 3;
+  const int t_lo = rank * n_out_tiles / LM_CLUSTER, t_hi = (rank + 1) * n_out_tiles / LM_CLUSTER;
+  const int s_first = rank * (LM_SEQ / LM_CLUSTER);
+
   // ---- what the later phases read is asked into L2 now (128-byte lines) -------------------------------------------------
   {
-    const char* pS = reinterpret_cast<const char*>(p.S + ((size_t)l * B + b0) * G * r);
-    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * G * r * 4; o += (size_t)LM_THREADS * 128)
+    const char* pS = reinterpret_cast<const char*>(p.S + ((size_t)l * B + b0 + s_first) * G * r);
+    const int ns4 = max(0, min(LM_SEQ / LM_CLUSTER, nseq - s_first));
+    for (size_t o = (size_t)tid * 128; o < (size_t)ns4 * G * r * 4; o += (size_t)LM_THREADS * 128)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(pS + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * d_out * 2; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(yl) + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)d_out * G * 2; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Al) + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)r * d_in * 2; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Bl) + o));
-    for (size_t o = (size_t)tid * 128; o < (size_t)nseq * d_in * 2; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(xl) + o));
+    const char* pA = reinterpret_cast<const char*>(Al + (size_t)t_lo * 8 * G);
+    for (size_t o = (size_t)tid * 128; o < (size_t)(t_hi - t_lo) * 8 * G * 2; o += (size_t)LM_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(pA + o));
+    for (int s = 0; s < nseq; ++s) {
+      const char* py = reinterpret_cast<const char*>(yl + (size_t)s * d_out + (size_t)t_lo * 8);
+      for (size_t o = (size_t)tid * 128; o < (size_t)(t_hi - t_lo) * 16; o += (size_t)LM_THREADS * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(py + o));
+    }
   }
 
-  // ---- u = X B^T -------------------------------------------------------------------------------------------------------
+  // ---- phase 1: u (this CTA's slice of d_in) ------------------------------------------------------------------------------
   {
-    const int n_pairs = d_in >> 5;                              // 32 contraction values per pair of mma steps
     const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    const int np = p_hi - p_lo;
     for (int item = warp; item < n_tiles * KS; item += LM_WARPS) {
       const int tile = item % n_tiles, ks = item / n_tiles;
-      const int s_lo = ks * n_pairs / KS, s_hi = (ks + 1) * n_pairs / KS;
+      const int s_lo = p_lo + ks * np / KS, s_hi = p_lo + (ks + 1) * np / KS;
       const __nv_bfloat16* wrow = Bl + (size_t)(tile * 8 + qrow) * d_in + qcol * 8;
       const __nv_bfloat16* xlo = xl + (size_t)qrow * d_in + qcol * 8;
       const __nv_bfloat16* xhi = xlo + (size_t)8 * d_in;
@@ -246,7 +267,7 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
           }
         }
       }
-      float* dst = u + ((size_t)ks * LM_SEQ + qrow) * r + tile * 8 + 2 * qcol;
+      float* dst = u_part + ((size_t)ks * LM_SEQ + qrow) * r + tile * 8 + 2 * qcol;
       dst[0] = c[0];
       dst[1] = c[1];
       dst[8 * r] = c[2];
@@ -254,50 +275,86 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
     }
   }
   __syncthreads();
-  // ---- w = S u (fp32), split into two bf16 terms: a warp per sequence, a lane per state row ---------------------------
-  for (int s = warp; s < LM_SEQ; s += LM_WARPS) {
-    for (int g = lane; g < G; g += 32) {
-      float acc = 0.f;
-      if (s < nseq) {
-        const float* Srow = p.S + (((size_t)l * B + b0 + s) * G + g) * r;
-        for (int j = 0; j < r; j += 4) {
-          const float4 sv = *reinterpret_cast<const float4*>(Srow + j);
-          float uu[4];
+  for (int i = tid; i < LM_SEQ * r; i += LM_THREADS) {
+    float t = u_part[i];
+    for (int ks = 1; ks < KS; ++ks) t += u_part[(size_t)ks * LM_SEQ * r + i];
+    u_loc[i] = t;
+  }
+  cluster.sync();                                              // every CTA's share of u is in its shared memory
+
+  // ---- phase 2: w = S u for this CTA's four sequences (a warp per sequence, a lane per state row) -----------------------
+  {
+    const float* u_rem[LM_CLUSTER];
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            float t = u[(size_t)s * r + j + k];
-            for (int ks = 1; ks < KS; ++ks) t += u[((size_t)ks * LM_SEQ + s) * r + j + k];
-            uu[k] = t;
+    for (int c = 0; c < LM_CLUSTER; ++c) u_rem[c] = cluster.map_shared_rank(u_loc, c);
+    for (int sq = warp; sq < LM_SEQ / LM_CLUSTER; sq += LM_WARPS) {
+      const int s = s_first + sq;
+      for (int g = lane; g < G; g += 32) {
+        float acc = 0.f;
+        if (s < nseq) {
+          const float* Srow = p.S + (((size_t)l * B + b0 + s) * G + g) * r;
+          for (int j0 = 0; j0 < r; j0 += 32) {                  // eight 16-byte loads of the state row in flight
+            float4 sv[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              sv[i] = (j0 + 4 * i < r) ? *reinterpret_cast<const float4*>(Srow + j0 + 4 * i)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int j = j0 + 4 * i;
+              if (j < r) {
+                float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < LM_CLUSTER; ++c) {           // the same order in every CTA
+                  const float4 t = *reinterpret_cast<const float4*>(u_rem[c] + (size_t)s * r + j);
+                  uu.x += t.x; uu.y += t.y; uu.z += t.z; uu.w += t.w;
+                }
+                acc = fmaf(sv[i].x, uu.x, acc);
+                acc = fmaf(sv[i].y, uu.y, acc);
+                acc = fmaf(sv[i].z, uu.z, acc);
+                acc = fmaf(sv[i].w, uu.w, acc);
+              }
+            }
           }
-          acc = fmaf(sv.x, uu[0], acc);
-          acc = fmaf(sv.y, uu[1], acc);
-          acc = fmaf(sv.z, uu[2], acc);
-          acc = fmaf(sv.w, uu[3], acc);
         }
+        const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
+        w_hi[s * G + g] = hi;
+        w_lo[s * G + g] = __float2bfloat16_rn(acc - __bfloat162float(hi));
       }
-      const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-      w_hi[s * G + g] = hi;
-      w_lo[s * G + g] = __float2bfloat16_rn(acc - __bfloat162float(hi));
     }
   }
-  __syncthreads();
-  // ---- y += w A^T : column tiles of 8 outputs, four per iteration so that a row's 64 bytes of y move together ---------
+  cluster.sync();                                              // every CTA's four rows of w are in its shared memory
+  // gather the other CTAs' rows of w (16 x G bf16 twice: a few KB)
+  {
+    const int per_cta = (LM_SEQ / LM_CLUSTER) * G;               // elements of w_hi (and of w_lo) a CTA produced
+    for (int c = 0; c < LM_CLUSTER; ++c) {
+      if (c == rank) continue;
+      const __nv_bfloat16* rh = cluster.map_shared_rank(w_hi, c) + c * per_cta;
+      const __nv_bfloat16* rl = cluster.map_shared_rank(w_lo, c) + c * per_cta;
+      for (int i = tid * 8; i < per_cta; i += LM_THREADS * 8) {
+        *reinterpret_cast<uint4*>(w_hi + c * per_cta + i) = *reinterpret_cast<const uint4*>(rh + i);
+        *reinterpret_cast<uint4*>(w_lo + c * per_cta + i) = *reinterpret_cast<const uint4*>(rl + i);
+      }
+    }
+  }
+  cluster.sync();                                              // remote reads done: peers may overwrite or exit
+
+  // ---- phase 3: y += w A^T for this CTA's share of the outputs, four column tiles per iteration ---------------------------
   {
     const int kp = G >> 5;                                      // pairs of mma steps along G
     const bool wr_lo = lo_ok && (active == nullptr || active[b0 + qrow] != 0);
     const bool wr_hi = hi_ok && (active == nullptr || active[b0 + qrow + 8] != 0);
-    const int n_out_tiles = d_out >> 3;
     // the w fragments of the first 32 state rows do not depend on the output tile
     const uint4 wh_l = *reinterpret_cast<const uint4*>(w_hi + qrow * G + qcol * 8);
     const uint4 wh_h = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + qcol * 8);
     const uint4 wl_l = *reinterpret_cast<const uint4*>(w_lo + qrow * G + qcol * 8);
     const uint4 wl_h = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + qcol * 8);
-    for (int t0 = warp * 4; t0 < n_out_tiles; t0 += LM_WARPS * 4) {
+    for (int t0 = t_lo + warp * 4; t0 < t_hi; t0 += LM_WARPS * 4) {
       uint4 aw[4];
       uint32_t yl4[4], yh4[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        if (t0 + q < n_out_tiles) {
+        if (t0 + q < t_hi) {
           const int i0 = (t0 + q) * 8;
           aw[q] = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + qcol * 8));
           yl4[q] = wr_lo ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
@@ -306,7 +363,7 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        if (t0 + q >= n_out_tiles) break;
+        if (t0 + q >= t_hi) break;
         const int i0 = (t0 + q) * 8;
         float c[4] = {0.f, 0.f, 0.f, 0.f};
         lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw[q].x, aw[q].y);
@@ -344,11 +401,13 @@ k_lora_apply_mma(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const 
 cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* A, const void* Bm, const void* x,
                                     void* y, const uint8_t* active, int d_in, int d_out, cudaStream_t st) {
   const PtencDev& p = c->dev;
-  // tensor-core path: bf16, r a multiple of 8, G and d_in multiples of 32, d_out a multiple of 8
-  if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && (d_out & 7) == 0 &&
-      lr_mma_smem(p.G, p.r) <= 48 * 1024) {
+  // tensor-core path: bf16, r a multiple of 8, G and d_in multiples of 32 (d_in at least 128: a slice per CTA of the
+  // cluster), d_out a multiple of 8
+  if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && d_in >= 128 &&
+      (d_out & 7) == 0 && lr_mma_smem(p.G, p.r) <= 48 * 1024 &&
+      (long long)nl * ((p.B + LM_SEQ - 1) / LM_SEQ) <= 65535) {
     const int nb = (p.B + LM_SEQ - 1) / LM_SEQ;
-    k_lora_apply_mma<<<nl * nb, LM_THREADS, lr_mma_smem(p.G, p.r), st>>>(
+    k_lora_apply_cluster<<<dim3(LM_CLUSTER, nl * nb), LM_THREADS, lr_mma_smem(p.G, p.r), st>>>(
         p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, active,
         d_in, d_out);
     c->launches++;

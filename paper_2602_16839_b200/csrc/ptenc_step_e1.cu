@@ -19,6 +19,9 @@ constexpr int RE_WARPS = 8;                // (layer, sequence) pairs per CTA
 __global__ void __launch_bounds__(RE_WARPS * 32)
 k_ring_e1(PtencDev p, int l0, int nl, const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
           const uint8_t* __restrict__ active) {
+  // the attention launch behind this kernel may become resident and run its set-up now; it waits for this whole
+  // grid before it reads anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * RE_WARPS + (threadIdx.x >> 5);
   if (item >= nl * p.B) return;
