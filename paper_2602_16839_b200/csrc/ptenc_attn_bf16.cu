@@ -686,25 +686,59 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       consumer_sync(NCONS);
       if (misc[1]) {
         __threadfence();
-        for (int idx = tid; idx < 8 * D; idx += NCONS) {
-          const int r = idx / D, d = idx - r * D;
-          if (r >= g) continue;
-          float mt = -INFINITY;
-          for (long long c = c_first; c <= c_last; ++c) {
-            const int slot = 2 * (int)c + (c == c_first ? 1 : 0);
-            mt = fmaxf(mt, __ldcg(&p.part_ml[slot * 16 + r]));
+        // NCONS / 8 threads per query-head row, each with every TPR-th output dim.  The partials sit in L2: the loads
+        // of two parts (a unit is rarely split further) (their m, l and this thread's share of the accumulators) are issued together, so the
+        // combine costs two memory round trips whatever the number of outputs -- it is the tail of the launch.
+        constexpr int TPR = NCONS / 8;
+        constexpr int PB = 2;                                   // parts whose loads are in flight together
+        constexpr int DPT = (D + TPR - 1) / TPR;
+        const int r = tid / TPR, d0 = tid - r * TPR;
+        float mrun = -INFINITY, lrun = 0.f;
+        float acc[DPT];
+#pragma unroll
+        for (int i = 0; i < DPT; ++i) acc[i] = 0.f;
+        for (long long c0 = c_first; c0 <= c_last; c0 += PB) {
+          float mw[PB], lw[PB], pa[PB][DPT];
+#pragma unroll
+          for (int u = 0; u < PB; ++u) {
+            const long long c = c0 + u;
+            const bool okc = c <= c_last;
+            const int slot = okc ? 2 * (int)c + (c == c_first ? 1 : 0) : 0;
+            mw[u] = okc ? __ldcg(&p.part_ml[slot * 16 + r]) : -INFINITY;
+            lw[u] = okc ? __ldcg(&p.part_ml[slot * 16 + 8 + r]) : 0.f;
+#pragma unroll
+            for (int i = 0; i < DPT; ++i) {
+              const int d = d0 + i * TPR;
+              pa[u][i] = (okc && d < D) ? __ldcg(&p.part_acc[((size_t)slot * 8 + r) * D + d]) : 0.f;
+            }
           }
-          float lt = 0.f, acc = 0.f;
-          for (long long c = c_first; c <= c_last; ++c) {
-            const int slot = 2 * (int)c + (c == c_first ? 1 : 0);
-            const float mw = __ldcg(&p.part_ml[slot * 16 + r]);
-            const float wg = (mw == -INFINITY) ? 0.f : ex2(mw - mt);
-            lt = fmaf(wg, __ldcg(&p.part_ml[slot * 16 + 8 + r]), lt);
-            acc = fmaf(wg, __ldcg(&p.part_acc[((size_t)slot * 8 + r) * D + d]), acc);
+          float mnew = mrun;
+#pragma unroll
+          for (int u = 0; u < PB; ++u) mnew = fmaxf(mnew, mw[u]);
+          if (c0 != c_first) {                                  // more parts than one batch: rescale what is summed so far
+            const float sc = (mrun == -INFINITY) ? 0.f : ex2(mrun - mnew);
+            lrun *= sc;
+#pragma unroll
+            for (int i = 0; i < DPT; ++i) acc[i] *= sc;
           }
-          out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc / lt);
-          if (lse != nullptr && d == 0) lse[orow0 + r] = (mt + log2f(lt)) * 0.6931471805599453f;
-          if (SCORE && d == 0) p.lse2[((size_t)(l0 + li) * B + b) * p.Hq + (size_t)h * g + r] = mt + log2f(lt);
+#pragma unroll
+          for (int u = 0; u < PB; ++u) {
+            const float wg = (mw[u] == -INFINITY) ? 0.f : ex2(mw[u] - mnew);
+            lrun = fmaf(wg, lw[u], lrun);
+#pragma unroll
+            for (int i = 0; i < DPT; ++i) acc[i] = fmaf(wg, pa[u][i], acc[i]);
+          }
+          mrun = mnew;
+        }
+        if (r < g) {
+#pragma unroll
+          for (int i = 0; i < DPT; ++i) {
+            const int d = d0 + i * TPR;
+            if (d < D) out[(orow0 + r) * D + d] = __float2bfloat16_rn(acc[i] / lrun);
+          }
+          if (lse != nullptr && d0 == 0) lse[orow0 + r] = (mrun + log2f(lrun)) * 0.6931471805599453f;
+          if (SCORE && d0 == 0)
+            p.lse2[((size_t)(l0 + li) * B + b) * p.Hq + (size_t)h * g + r] = mrun + log2f(lrun);
         }
         if (SCORE && tid == 0) p.pending[(size_t)(l0 + li) * B + b] = 1;
       }

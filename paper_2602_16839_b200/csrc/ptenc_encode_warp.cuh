@@ -14,7 +14,8 @@
 
 constexpr int ENCW_MAX_VEC = 4;        // 16-byte vectors of a row held per lane: d_kv <= 32 * 4 * 8 = 1024
 constexpr int ENCW_MAX_RB = 4;         // 32-wide blocks of the rank: r <= 128
-constexpr int ENCW_JB = 4;             // output rows whose weights are in flight together
+constexpr int ENCW_W_VEC = 8;          // 16-byte vectors of EACH weight matrix a lane keeps in flight: with NV vectors
+                                       // per row and lane, 8 / NV output rows are requested per memory round trip
 
 __device__ __forceinline__ float encw_dot8(const uint4& w, const uint4& x) {
   const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&w);
@@ -34,14 +35,16 @@ __host__ __device__ inline bool encw_shape_ok(int G, int r, int d_kv) {
   return (r & 7) == 0 && r <= 32 * ENCW_MAX_RB && (d_kv & 31) == 0 && d_kv <= 256 * ENCW_MAX_VEC && G >= 1 && G <= 128;
 }
 
-// rowK, rowV: the evicted token's key and value rows [d_kv] bf16 (16-byte aligned).  The whole warp must call.
-__device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t lb, const __nv_bfloat16* rowK,
-                                              const __nv_bfloat16* rowV, int lane) {
+// NV = 16-byte vectors of a row per lane (2 or 4: d_kv <= 512, 1024).
+template <int NV>
+__device__ __forceinline__ void encw_fold_row_t(const PtencDev& p, int l, size_t lb, const __nv_bfloat16* rowK,
+                                                const __nv_bfloat16* rowV, int lane) {
+  constexpr int ENCW_JB = ENCW_W_VEC / NV;                   // 4 or 2 output rows per batch
   const int G = p.G, r = p.r, d_kv = p.d_kv;
   const int nv = d_kv >> 3;                                  // 16-byte vectors per row
-  uint4 xk[ENCW_MAX_VEC], xv[ENCW_MAX_VEC];
+  uint4 xk[NV], xv[NV];
 #pragma unroll
-  for (int u = 0; u < ENCW_MAX_VEC; ++u) {
+  for (int u = 0; u < NV; ++u) {
     const int v = lane + 32 * u;
     xk[u] = make_uint4(0u, 0u, 0u, 0u);
     xv[u] = xk[u];
@@ -59,14 +62,14 @@ __device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t l
   float ka[ENCW_MAX_RB], va[ENCW_MAX_RB];
 #pragma unroll
   for (int jb = 0; jb < ENCW_MAX_RB; ++jb) { ka[jb] = 0.f; va[jb] = 0.f; }
-  for (int j0 = 0; j0 < r; j0 += ENCW_JB) {                  // r is a multiple of 8
-    uint4 wk[ENCW_JB][ENCW_MAX_VEC], wv[ENCW_JB][ENCW_MAX_VEC];
+  for (int j0 = 0; j0 < r; j0 += ENCW_JB) {                  // r is a multiple of 8; a batch may run past r
+    uint4 wk[ENCW_JB][NV], wv[ENCW_JB][NV];
 #pragma unroll
     for (int jj = 0; jj < ENCW_JB; ++jj) {
 #pragma unroll
-      for (int u = 0; u < ENCW_MAX_VEC; ++u) {
+      for (int u = 0; u < NV; ++u) {
         const int v = lane + 32 * u;
-        if (v < nv) {
+        if (v < nv && j0 + jj < r) {
           wk[jj][u] = __ldg(reinterpret_cast<const uint4*>(Wk + (size_t)(j0 + jj) * d_kv + (size_t)v * 8));
           wv[jj][u] = __ldg(reinterpret_cast<const uint4*>(Wv + (size_t)(j0 + jj) * d_kv + (size_t)v * 8));
         }
@@ -74,9 +77,10 @@ __device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t l
     }
 #pragma unroll
     for (int jj = 0; jj < ENCW_JB; ++jj) {
+      if (j0 + jj >= r) break;                               // uniform over the warp
       float sk = 0.f, sv = 0.f;
 #pragma unroll
-      for (int u = 0; u < ENCW_MAX_VEC; ++u) {
+      for (int u = 0; u < NV; ++u) {
         if (lane + 32 * u < nv) {
           sk += encw_dot8(wk[jj][u], xk[u]);
           sv += encw_dot8(wv[jj][u], xv[u]);
@@ -176,4 +180,11 @@ __device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t l
       }
     }
   }
+}
+
+// rowK, rowV: the evicted token's key and value rows [d_kv] bf16 (16-byte aligned).  The whole warp must call.
+__device__ __forceinline__ void encw_fold_row(const PtencDev& p, int l, size_t lb, const __nv_bfloat16* rowK,
+                                              const __nv_bfloat16* rowV, int lane) {
+  if (p.d_kv <= 512) encw_fold_row_t<2>(p, l, lb, rowK, rowV, lane);
+  else encw_fold_row_t<4>(p, l, lb, rowK, rowV, lane);
 }
