@@ -248,6 +248,7 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   d.tickets = reinterpret_cast<int*>(base + lay.tickets);
   d.part_slots = PART_SLOTS;
   d.status = reinterpret_cast<int*>(base + lay.status);
+  d.work = d.status + 4;                               // same 64-byte block as the status word
   d.policy = cfg->policy; d.recent = cfg->recent; d.wb = 0;
   d.slot_tok = nullptr; d.score = nullptr; d.live_bits = nullptr; d.logits = nullptr; d.lse2 = nullptr;
   d.pending = nullptr; d.fq = nullptr; d.fq_head = nullptr; d.fq_count = nullptr; d.ev_tok = nullptr; d.ev_slot = nullptr;

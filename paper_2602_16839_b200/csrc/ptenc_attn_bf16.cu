@@ -5,14 +5,15 @@
 // is read once per step and there is no reuse between steps.
 //
 // Design
-//  * Persistent grid, one CTA per SM.  The work is the flat list of K/V tiles (32 tokens at head_dim 128, 64 at
-//    head_dim 64) of every (layer, sequence, KV head) unit that has live tokens; CTA c takes the contiguous share
-//    [c*T/n, (c+1)*T/n) of the T tiles, so no SM idles in a tail wave whatever B*H_kv is (split-K at tile
-//    granularity, sized to the machine).
+//  * Persistent grid, one CTA per SM.  The work is the K/V tiles (32 tokens at head_dim 128, 64 at head_dim 64) of
+//    every (layer, sequence, KV head) unit that has live tokens, cut into work items: a whole unit, or -- when the
+//    call is small -- pieces of a unit, so that every CTA gets several items (split-K sized to the machine).  CTAs
+//    take items from a counter in global memory as they go: SMs do not stream at the same rate, and with fixed equal
+//    shares the slowest SM set the time of the launch.
 //  * A producer warp streams K and V tiles with TMA (cp.async.bulk.tensor, 128-byte swizzle; plain per-CTA loads
 //    of this GPU's own memory) into a ring of shared-memory stages guarded by full/empty mbarriers.
-//  * Each consumer warp owns whole tiles (tile n of the CTA goes to warp n mod NW, stage n mod STAGES; STAGES
-//    is a multiple of NW so a stage always has the same consumer warp and its full/empty barriers advance
+//  * Each consumer warp owns whole tiles (tile i of an item goes to warp i mod NW, which cycles through its own
+//    STAGES / NW pipeline stages, so a stage always has the same consumer warp and its full/empty barriers advance
 //    one phase per visit -- a warp can never be a phase ahead of a barrier it polls).  The two products run on
 //    warp-level bf16 mma (m16n8k16, fp32 accumulate) only to keep the FP32 pipes free, in transposed form so that
 //    all 16 rows of the mma carry data: S^T = K Q^T (rows = 16 tokens, columns = the g <= 8 query heads) and
@@ -168,7 +169,8 @@ struct Smem {
   static constexpr int OFF_ML = OFF_ACC + NW * 8 * ACC_STRIDE * 4;
   static constexpr int OFF_BAR = OFF_ML + NW * 16 * 4;
   static constexpr int OFF_MISC = OFF_BAR + (2 * STAGES + 4) * 8;
-  static constexpr int TOTAL = OFF_MISC + 64;
+  static constexpr int OFF_DESC = OFF_MISC + 64;            // two work-item descriptions of 16 ints
+  static constexpr int TOTAL = OFF_DESC + 128;
 };
 
 // ------------------------------------------------------------------------------------------------ kernel
@@ -197,9 +199,16 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   const uint32_t bar_qfull = bar_empty + STAGES * 8;
   const uint32_t bar_qempty = bar_qfull + 2 * 8;
   volatile int* misc = reinterpret_cast<volatile int*>(smem + SM::OFF_MISC);
-  // misc[0] abort flag, misc[1] last-arriver flag, misc[2] start entry, misc[4..5] start prefix (int64),
-  // misc[6..7] total tiles per head-sum (int64)
+  // misc[0] abort flag, misc[1] last-arriver flag, misc[8..9] verdict on the item in description slot 0 / 1
+  // (1 = work on it, 2 = stop)
+  volatile int* desc = reinterpret_cast<volatile int*>(smem + SM::OFF_DESC);
+  // description of a work item: [0] 1 = item, 2 = no more items; [1] layer of the call, [2] sequence, [3] KV head;
+  // [4..8] ring state and tile enumeration of the unit (head, count, pinned, t0, len2); [9] first tile of the piece
+  // in the unit's enumeration, [10] tiles of the piece; [11] pieces of the unit, [12] this piece, [13] first partial
+  // slot of the unit (split units only)
   __shared__ long long s_part[NTHREADS];
+  __shared__ int s_items[NTHREADS + 1];
+  __shared__ int s_split[NTHREADS + 1];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = p.W, B = p.B, Hkv = p.Hkv, g = p.g;
@@ -210,7 +219,8 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull + 8 * s, 1); mbar_init(bar_qempty + 8 * s, NW); }
-    misc[0] = 0; misc[1] = 0; misc[2] = -1; misc[4] = -1; misc[5] = -1;
+    misc[0] = 0; misc[1] = 0; misc[8] = 0; misc[9] = 0;
+    desc[0] = 0; desc[16] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < 2 * SM::Q_BYTES / 4; i += NTHREADS) reinterpret_cast<uint32_t*>(smem + SM::OFF_Q)[i] = 0u;
@@ -220,7 +230,13 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   // read before this point.  A no-op for an ordinary launch.
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  // ---- schedule: total tile count and this CTA's starting entry ------------------------------------
+  // ---- schedule ----------------------------------------------------------------------------------------------------
+  // Work items.  The tiles of a (layer, sequence, KV head) unit are one item, or -- when the call has too few tiles
+  // to give every CTA several items -- P pieces of about `piece` tiles each.  Items are numbered in (entry, head,
+  // piece) order and handed out at run time: a CTA that finishes an item takes the next number from a counter in
+  // global memory.  SMs do not all stream at the same rate (a fixed equal share left the slowest of them 10 % behind
+  // the median at the largest shapes), so the hand-out is dynamic; which CTA computes an item has no influence on
+  // the result.
   struct Raw { int head, count, sink, act; long long n; };
   // the ring words of one entry; every load is unconditional (index clamped) so that the loads of several entries
   // can be in flight together
@@ -262,6 +278,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     return en;
   };
   auto load_entry = [&](int e) -> Entry { return make_entry(fetch(e), e); };
+  // every thread takes a contiguous chunk of the entries; tiles, items and pieces of split units per chunk
   const int chunk = (n_ent + NTHREADS - 1) / NTHREADS;
   const int e_lo = min(tid * chunk, n_ent), e_hi = min(e_lo + chunk, n_ent);
   long long mine = 0;
@@ -275,31 +292,42 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   }
   s_part[tid] = mine;
   __syncthreads();
-  long long before = 0, total = 0;
-  for (int i = 0; i < NTHREADS; ++i) {
-    const long long v = s_part[i];
-    if (i < tid) before += v;
-    total += v;
-  }
+  long long total = 0;
+  for (int i = 0; i < NTHREADS; ++i) total += s_part[i];
   const long long T = total * Hkv;                     // tiles of the whole call
-  const long long n_cta = (T < (long long)gridDim.x) ? T : (long long)gridDim.x;
-  const bool has_tiles = (long long)blockIdx.x < n_cta;
-  const long long t_begin = has_tiles ? (long long)blockIdx.x * T / n_cta : 0;
-  const long long t_end = has_tiles ? (long long)(blockIdx.x + 1) * T / n_cta : 0;
-
-  // the thread whose chunk contains t_begin finds the entry
-  if (has_tiles && mine > 0 && before * Hkv <= t_begin && t_begin < (before + mine) * Hkv) {
-    long long pe = before;
-    int e = e_lo;
-    for (; e < e_hi; ++e) {
-      const int nt = load_entry(e).nt;
-      if (t_begin < (pe + nt) * Hkv) break;
-      pe += nt;
+  // piece size: about `bal` items per CTA when the call is small; a unit is never cut finer than 8 tiles.  With
+  // bal <= part_slots / (2 gridDim) the pieces of split units always fit the partial slots: a unit is split only if
+  // it has more than `piece` tiles, so there are at most T / piece + T / piece <= 2 bal gridDim such pieces.
+  long long bal = p.part_slots / (2 * (long long)gridDim.x);
+  bal = bal < 1 ? 1 : (bal > 4 ? 4 : bal);
+  long long piece_ll = (T + bal * gridDim.x - 1) / (bal * gridDim.x);
+  const int piece = (int)(piece_ll < 8 ? 8 : (piece_ll > (1 << 24) ? (1 << 24) : piece_ll));
+  auto pieces_of = [&](int nt) -> int { return nt <= 0 ? 0 : (nt + piece - 1) / piece; };
+  {
+    int items = 0, split = 0;
+    for (int e = e_lo; e < e_hi; ++e) {                       // the ring words are in L1 now
+      const int pc = pieces_of(load_entry(e).nt);
+      items += Hkv * pc;
+      if (pc > 1) split += Hkv * pc;
     }
-    misc[2] = e;
-    *reinterpret_cast<volatile long long*>(&misc[4]) = pe;
+    s_items[tid] = items;
+    s_split[tid] = split;
   }
   __syncthreads();
+  {
+    int bi = 0, bs = 0, ti = 0, ts = 0;
+    for (int i = 0; i < NTHREADS; ++i) {
+      const int vi = s_items[i], vs = s_split[i];
+      if (i < tid) { bi += vi; bs += vs; }
+      ti += vi; ts += vs;
+    }
+    __syncthreads();
+    s_items[tid] = bi;                                        // exclusive prefixes; the totals go last
+    s_split[tid] = bs;
+    if (tid == 0) { s_items[NTHREADS] = ti; s_split[NTHREADS] = ts; }
+  }
+  __syncthreads();
+  const int n_items = s_items[NTHREADS];
 
   if (warp > NW) {
     // ================================================================ encoder warps (see the file header)
@@ -319,91 +347,155 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     }
     return;
   }
-  if (!has_tiles) return;                              // also when the call has no live token at all (T == 0)
-  const int e_start = misc[2];
-  const long long pe_start = *reinterpret_cast<volatile long long*>(&misc[4]);
-  if (e_start < 0 || e_start >= n_ent || pe_start < 0 || pe_start * Hkv > t_begin) {   // uniform over the CTA
-    if (tid == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
-    return;
-  }
-
-  // Every warp walks the same sequence of units: (entry e, head h) with unit tile interval
-  // [ub, ub + nt) in the flat list, clipped to [t_begin, t_end).
-  int e = e_start;
-  Entry en = load_entry(e);
-  int h = (int)((t_begin - pe_start * Hkv) / en.nt);
-  long long ub = pe_start * Hkv + (long long)h * en.nt;
-  Entry nxt;                                             // prefetched entry e + 1
-  nxt.nt = 0; nxt.head = nxt.count = nxt.sink = nxt.t0 = nxt.len2 = 0;
-  if (e + 1 < n_ent) nxt = load_entry(e + 1);
-
-  auto advance = [&]() {                                 // to the next unit with tiles
-    ub += en.nt;
-    if (++h < Hkv) return;
-    h = 0;
-    do {
-      ++e;
-      en = nxt;
-      if (e + 1 < n_ent) nxt = load_entry(e + 1); else nxt.nt = 0;
-    } while (e < n_ent && en.nt == 0);
-  };
 
   const float sl2 = 1.4426950408889634f / sqrtf((float)D);
-  const uint32_t policy_dummy = 0; (void)policy_dummy;
+  // Pipeline stages belong to consumer warps: warp w owns stages [w SPW, (w + 1) SPW) and takes the tiles i = w
+  // (mod NW) of every item, so a stage's barriers always have the same consumer, and which warp sums which tiles of
+  // an item does not depend on what the CTA worked on before (results are reproducible bit for bit).
+  constexpr int SPW = STAGES / NW;
 
   if (warp == NW) {
-    // ================================================================ producer warp (one lane issues)
-    if (lane == 0) {
-      uint32_t n = 0;          // tiles issued by this CTA
-      uint32_t useq = 0;       // units visited
-      bool aborted = false;
-      const long long rows_total = (long long)p.L * B * Hkv * W;
-      while (ub < t_end && e < n_ent && !aborted) {
-        const long long lo = ub > t_begin ? ub : t_begin;
-        const long long hi = (ub + en.nt) < t_end ? (ub + en.nt) : t_end;
+    // ================================================================ producer warp
+    // All lanes look an item up (ballots and scans over the chunk prefixes); lane 0 owns the barriers and issues.
+    uint32_t kw[NW];                                         // tiles issued so far for each consumer warp
+#pragma unroll
+    for (int w = 0; w < NW; ++w) kw[w] = 0;
+    uint32_t useq = 0;                                       // items handed to the consumers
+    bool aborted = false;
+    const long long rows_total = (long long)p.L * B * Hkv * W;
+    while (!aborted) {
+      int item = 0;
+      if (lane == 0) item = atomicAdd(p.work, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      const uint32_t ubuf = useq & 1;
+      volatile int* dsc = desc + ubuf * 16;
+      if (item >= n_items) {
+        // nothing left: tell the consumers, and the CTA that makes the very last grab of the launch rewinds the
+        // counter for the next one
+        if (lane == 0) {
+          if (item == n_items + (int)gridDim.x - 1) *p.work = 0;
+          if (mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) {
+            dsc[0] = 2;
+            mbar_arrive(bar_qfull + 8 * ubuf);
+          } else {
+            aborted = true;
+          }
+        }
+        break;
+      }
+      // ---- which (entry, head, piece) is item number `item` --------------------------------------------------
+      int tch = -1;
+      for (int base = 0; base < NTHREADS; base += 32) {
+        const int idx = base + lane;
+        const bool hit = idx < NTHREADS && s_items[idx] <= item && item < s_items[idx + 1];
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m != 0) { tch = base + __ffs(m) - 1; break; }
+      }
+      Entry en;
+      en.head = en.count = en.sink = en.nt = en.t0 = en.len2 = 0;
+      int e = -1, rem = 0, split_before = 0;
+      if (tch >= 0) {
+        rem = item - s_items[tch];
+        split_before = s_split[tch];
+        const int ce_lo = min(tch * chunk, n_ent), ce_hi = min(ce_lo + chunk, n_ent);
+        for (int base = ce_lo; base < ce_hi && e < 0; base += 32) {
+          const int ee = base + lane;
+          Entry le = load_entry(ee < ce_hi ? ee : -1);
+          const int pc = pieces_of(le.nt);
+          const int it = Hkv * pc, sp = pc > 1 ? it : 0;
+          int it_inc = it, sp_inc = sp;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xffffffffu, it_inc, o), c = __shfl_up_sync(0xffffffffu, sp_inc, o);
+            if (lane >= o) { it_inc += a; sp_inc += c; }
+          }
+          const bool hit = it > 0 && it_inc - it <= rem && rem < it_inc;
+          const unsigned m = __ballot_sync(0xffffffffu, hit);
+          if (m != 0) {
+            const int src = __ffs(m) - 1;
+            e = base + src;
+            rem -= __shfl_sync(0xffffffffu, it_inc - it, src);
+            split_before += __shfl_sync(0xffffffffu, sp_inc - sp, src);
+            en.head = __shfl_sync(0xffffffffu, le.head, src);
+            en.count = __shfl_sync(0xffffffffu, le.count, src);
+            en.sink = __shfl_sync(0xffffffffu, le.sink, src);
+            en.nt = __shfl_sync(0xffffffffu, le.nt, src);
+            en.t0 = __shfl_sync(0xffffffffu, le.t0, src);
+            en.len2 = __shfl_sync(0xffffffffu, le.len2, src);
+          } else {
+            rem -= __shfl_sync(0xffffffffu, it_inc, 31);
+            split_before += __shfl_sync(0xffffffffu, sp_inc, 31);
+          }
+        }
+      }
+      const int P = pieces_of(en.nt);
+      if (e < 0 || P <= 0 || rem < 0 || rem >= Hkv * P) {      // uniform over the warp
+        if (lane == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+        aborted = true;
+        break;
+      }
+      const int h = rem / P, k = rem - h * P;
+      const int iu_lo = (int)((long long)k * en.nt / P), iu_hi = (int)((long long)(k + 1) * en.nt / P);
+      const int n_mine = iu_hi - iu_lo;
+      const int slot_base = P > 1 ? split_before + h * P : 0;
+      if (n_mine <= 0 || slot_base + P > p.part_slots) {
+        if (lane == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+        aborted = true;
+        break;
+      }
+      if (lane == 0) {
         const int li = e / B, b = e - li * B;
         const size_t lb = (size_t)(l0 + li) * B + b;
-        if (h < 0 || h >= Hkv || hi <= lo) { atomicOr(p.status, PTENC_ST_BAD_SCHEDULE); aborted = true; break; }
-        // Q rows of the unit
-        {
-          const uint32_t ubuf = useq & 1;
-          if (!mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) { aborted = true; break; }
+        // the item's description and the Q rows of its unit
+        if (!mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) { aborted = true; }
+        if (!aborted) {
+          dsc[1] = li; dsc[2] = b; dsc[3] = h; dsc[4] = en.head; dsc[5] = en.count; dsc[6] = en.sink;
+          dsc[7] = en.t0; dsc[8] = en.len2; dsc[9] = iu_lo; dsc[10] = n_mine; dsc[11] = P; dsc[12] = k;
+          dsc[13] = slot_base; dsc[0] = 1;
           const uint32_t qbytes = (uint32_t)(g * D * 2);
           mbar_expect_tx(bar_qfull + 8 * ubuf, qbytes);
           bulk_load(smem_base + SM::OFF_Q + ubuf * SM::Q_BYTES,
                     q + (((size_t)li * B + b) * p.Hq + (size_t)h * g) * D, qbytes, bar_qfull + 8 * ubuf);
-        }
-        const long long row0 = ((long long)lb * Hkv + h) * W;
-        for (long long t = lo; t < hi; ++t, ++n) {
-          const int iu = (int)(t - ub);                  // i-th tile of the unit
-          const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
-          const uint32_t s = n % STAGES;
-          const long long yy = row0 + (long long)j * TILE_N;
-          if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
-            atomicOr(p.status, PTENC_ST_BAD_INDEX); aborted = true; break;
-          }
-          if (!mbar_wait(bar_empty + 8 * s, ((n / STAGES) & 1) ^ 1)) { aborted = true; break; }
-          const uint32_t dst = smem_base + s * SM::STAGE_BYTES;
-          const uint32_t fb = bar_full + 8 * s;
-          mbar_expect_tx(fb, SM::STAGE_BYTES);
-          const int y = (int)yy;
+          const long long row0 = ((long long)lb * Hkv + h) * W;
+          for (int i0 = 0; i0 < n_mine && !aborted; i0 += NW) {
 #pragma unroll
-          for (int hf = 0; hf < D / 64; ++hf) {
-            tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
-            tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
+            for (int w = 0; w < NW; ++w) {
+              if (i0 + w >= n_mine || aborted) continue;
+              const int iu = iu_lo + i0 + w;                 // tile of the unit, in its enumeration order
+              const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
+              const uint32_t s = w * SPW + kw[w] % SPW;
+              const long long yy = row0 + (long long)j * TILE_N;
+              if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
+                atomicOr(p.status, PTENC_ST_BAD_INDEX); aborted = true; continue;
+              }
+              if (!mbar_wait(bar_empty + 8 * s, ((kw[w] / SPW) & 1) ^ 1)) { aborted = true; continue; }
+              const uint32_t dst = smem_base + s * SM::STAGE_BYTES;
+              const uint32_t fb = bar_full + 8 * s;
+              mbar_expect_tx(fb, SM::STAGE_BYTES);
+              const int y = (int)yy;
+#pragma unroll
+              for (int hf = 0; hf < D / 64; ++hf) {
+                tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
+                tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
+              }
+              kw[w] += 1;
+            }
           }
         }
-        ++useq;
-        advance();
       }
-      if (aborted) {
-        atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
-        misc[0] = 1;
-        // copies still in flight must land before the CTA's shared memory goes away
-        const uint32_t back = n < (uint32_t)STAGES ? n : (uint32_t)STAGES;
+      aborted = __shfl_sync(0xffffffffu, aborted ? 1 : 0, 0) != 0;
+      ++useq;
+    }
+    if (lane == 0 && aborted) {
+      atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
+      misc[0] = 1;
+      // copies still in flight must land before the CTA's shared memory goes away
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const uint32_t back = kw[w] < (uint32_t)SPW ? kw[w] : (uint32_t)SPW;
         for (uint32_t i = 0; i < back; ++i) {
-          const uint32_t nn = n - 1 - i;
-          (void)mbar_wait(bar_full + 8 * (nn % STAGES), (nn / STAGES) & 1);
+          const uint32_t kk = kw[w] - 1 - i;
+          (void)mbar_wait(bar_full + 8 * (w * SPW + kk % SPW), (kk / SPW) & 1);
         }
       }
     }
@@ -413,25 +505,33 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   // ================================================================== consumer warps
   const int qr = lane >> 2;          // row of the fragment = query head within the group
   const int qc = lane & 3;
-  uint32_t n = 0;                    // CTA tile sequence number of the unit's first tile
+  uint32_t kq = 0;                   // tiles this warp has consumed
   uint32_t useq = 0;
+  // The next item is announced by one thread: it waits for the item's barrier and posts a verdict that everybody reads
+  // behind a consumer barrier, so that the warps agree on going on or stopping even when a wait runs out.
+  auto announce = [&](uint32_t us) {
+    const uint32_t ub2 = us & 1;
+    int v = 2;
+    if (misc[0] == 0 && mbar_wait(bar_qfull + 8 * ub2, (us >> 1) & 1)) v = desc[ub2 * 16];
+    else { atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT); misc[0] = 1; }
+    misc[8 + ub2] = v;
+  };
+  if (tid == 0) announce(0);
+  consumer_sync(NCONS);
 
-  while (ub < t_end && e < n_ent) {
-    const long long lo = ub > t_begin ? ub : t_begin;
-    const long long hi = (ub + en.nt) < t_end ? (ub + en.nt) : t_end;
-    const int n_mine = (int)(hi - lo);
-    const int li = e / B, b = e - li * B;
-    const int head = en.head, count = en.count, sink = en.sink, cap = W - en.sink;
+  while (true) {
+    const uint32_t ubuf = useq & 1;
+    if (misc[8 + ubuf] != 1) break;                          // no more items (or a wait ran out): uniform over the CTA
+    (void)mbar_wait(bar_qfull + 8 * ubuf, (useq >> 1) & 1);  // completed already; orders this thread's reads behind it
+    volatile int* dsc = desc + ubuf * 16;
+    const int li = dsc[1], b = dsc[2], h = dsc[3];
+    const int head = dsc[4], count = dsc[5], sink = dsc[6], t0 = dsc[7], len2 = dsc[8];
+    const int iu_lo = dsc[9], n_mine = dsc[10], n_parts = dsc[11], piece_k = dsc[12], slot_base = dsc[13];
+    const int cap = W - sink;
 
     // ---- Q fragments (A operand, rows = heads; rows >= g are zero) ------------------------------------
     uint32_t qa[KSTEPS][2];
     {
-      const uint32_t ubuf = useq & 1;
-      if (misc[0] == 0 && !mbar_wait(bar_qfull + 8 * ubuf, (useq >> 1) & 1)) {
-        atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
-        misc[0] = 1;
-      }
-      __syncwarp();
       const uint8_t* qb = smem + SM::OFF_Q + ubuf * SM::Q_BYTES + qr * (D * 2) + qc * 4;
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -439,7 +539,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         qa[ks][1] = *reinterpret_cast<const uint32_t*>(qb + ks * 32 + 16);
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_qempty + 8 * ubuf);
+      if (lane == 0) mbar_arrive(bar_qempty + 8 * ubuf);     // the description and the Q rows have been read
     }
 
     // Transposed products, so that the 16 rows of the mma are always full: S^T = K Q^T (rows = tokens, columns = the
@@ -452,19 +552,17 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
 #pragma unroll
     for (int i = 0; i < DT; ++i) { oT[i][0] = 0.f; oT[i][1] = 0.f; oT[i][2] = 0.f; oT[i][3] = 0.f; }
 
-    int i0 = (int)((warp + NW - (n % NW)) % NW);
-    for (int i = i0; i < n_mine; i += NW) {
-      const uint32_t seq = n + i;
-      const uint32_t s = seq % STAGES;
-      const int iu = (int)(lo - ub) + i;
-      const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
+    for (int i = warp; i < n_mine; i += NW, ++kq) {
+      const uint32_t s = warp * SPW + kq % SPW;
+      const int iu = iu_lo + i;
+      const int j = iu < len2 ? t0 + iu : iu - len2;
       uint32_t lw0 = 0xffffffffu, lw1 = 0xffffffffu;        // liveness of the tile's slots (SCORE), requested early
       if (SCORE) {
         const unsigned int* lw = p.live_bits + ((size_t)(l0 + li) * B + b) * p.wb + ((j * TILE_N) >> 5);
         lw0 = lw[0];
         if (TILE_N > 32) lw1 = lw[1];
       }
-      if (misc[0] == 0 && !mbar_wait(bar_full + 8 * s, (seq / STAGES) & 1)) {
+      if (misc[0] == 0 && !mbar_wait(bar_full + 8 * s, (kq / SPW) & 1)) {
         atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
         misc[0] = 1;
       }
@@ -615,18 +713,14 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     }
     consumer_sync(NCONS);
 
-    const long long ue = ub + en.nt;
-    const bool whole = (lo == ub) && (hi == ue);
+    const bool whole = n_parts == 1;
     const size_t unit_id = ((size_t)(l0 + li) * B + b) * Hkv + h;
     const size_t orow0 = ((size_t)li * B + b) * p.Hq + (size_t)h * g;
-    int my_slot = 0;
-    if (!whole) my_slot = 2 * blockIdx.x + ((lo == ub) ? 1 : 0);
-    if (my_slot >= p.part_slots || h < 0 || h >= Hkv || n_mine <= 0) {      // uniform over the CTA
-      if (tid == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+    const int my_slot = slot_base + piece_k;                  // used by pieces of split units only
+    if (h < 0 || h >= Hkv || n_mine <= 0 || n_parts < 1 || (!whole && slot_base + n_parts > p.part_slots)) {
+      if (tid == 0) { atomicOr(p.status, PTENC_ST_BAD_SCHEDULE); announce(useq + 1); }   // uniform over the CTA
       consumer_sync(NCONS);
-      n += (uint32_t)(n_mine > 0 ? n_mine : 0);
       ++useq;
-      advance();
       continue;
     }
 
@@ -672,9 +766,6 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
 
     if (!whole) {
       // ---- split unit: publish the partial; the CTA that arrives last combines ---------------------------------
-      const long long c_first = ((ub + 1) * n_cta - 1) / T;
-      const long long c_last = (ue * n_cta - 1) / T;
-      const int n_parts = (int)(c_last - c_first + 1);
       __threadfence();
       consumer_sync(NCONS);
       if (tid == 0) {
@@ -687,8 +778,8 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       if (misc[1]) {
         __threadfence();
         // NCONS / 8 threads per query-head row, each with every TPR-th output dim.  The partials sit in L2: the loads
-        // of two parts (a unit is rarely split further) (their m, l and this thread's share of the accumulators) are issued together, so the
-        // combine costs two memory round trips whatever the number of outputs -- it is the tail of the launch.
+        // of two parts (their m, l and this thread's share of the accumulators) are issued together, so the combine
+        // of a unit in two pieces costs two memory round trips -- it is the tail of the launch.
         constexpr int TPR = NCONS / 8;
         constexpr int PB = 2;                                   // parts whose loads are in flight together
         constexpr int DPT = (D + TPR - 1) / TPR;
@@ -697,13 +788,13 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         float acc[DPT];
 #pragma unroll
         for (int i = 0; i < DPT; ++i) acc[i] = 0.f;
-        for (long long c0 = c_first; c0 <= c_last; c0 += PB) {
+        for (int c0 = 0; c0 < n_parts; c0 += PB) {
           float mw[PB], lw[PB], pa[PB][DPT];
 #pragma unroll
           for (int u = 0; u < PB; ++u) {
-            const long long c = c0 + u;
-            const bool okc = c <= c_last;
-            const int slot = okc ? 2 * (int)c + (c == c_first ? 1 : 0) : 0;
+            const int c = c0 + u;
+            const bool okc = c < n_parts;
+            const int slot = okc ? slot_base + c : slot_base;
             mw[u] = okc ? __ldcg(&p.part_ml[slot * 16 + r]) : -INFINITY;
             lw[u] = okc ? __ldcg(&p.part_ml[slot * 16 + 8 + r]) : 0.f;
 #pragma unroll
@@ -715,7 +806,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
           float mnew = mrun;
 #pragma unroll
           for (int u = 0; u < PB; ++u) mnew = fmaxf(mnew, mw[u]);
-          if (c0 != c_first) {                                  // more parts than one batch: rescale what is summed so far
+          if (c0 != 0) {                                        // more parts than one batch: rescale what is summed so far
             const float sc = (mrun == -INFINITY) ? 0.f : ex2(mrun - mnew);
             lrun *= sc;
 #pragma unroll
@@ -743,11 +834,9 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         if (SCORE && tid == 0) p.pending[(size_t)(l0 + li) * B + b] = 1;
       }
     }
-    consumer_sync(NCONS);       // merge buffers and misc[1] are free again
-
-    n += (uint32_t)n_mine;
+    if (tid == 0) announce(useq + 1);
+    consumer_sync(NCONS);       // merge buffers and misc[1] are free again; the verdict on the next item is posted
     ++useq;
-    advance();
   }
 }
 
@@ -1012,6 +1101,7 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   d.head = const_cast<int*>(head);
   d.count = const_cast<int*>(count);
   d.status = reinterpret_cast<int*>(sd->scratch + STATIC_OFF_STATUS);
+  d.work = reinterpret_cast<int*>(sd->scratch + STATIC_OFF_STATUS + 16);
   d.tickets = reinterpret_cast<int*>(sd->scratch + STATIC_OFF_TICKETS);
   d.part_ml = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ML);
   d.part_acc = reinterpret_cast<float*>(sd->scratch + STATIC_OFF_ACC);
@@ -1019,7 +1109,7 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   int grid = sd->sm_count * PTENC_ATTN_CTAS_PER_SM;
   if (2 * grid > STATIC_MAX_SLOTS) grid = STATIC_MAX_SLOTS / 2;
 
-  // The array keeps whatever the last call left: the status word and the tickets must start at zero.
+  // The array keeps whatever the last call left: the status word, the work counter and the tickets must start at zero.
   if (cudaMemsetAsync(sd->scratch, 0, STATIC_OFF_TICKETS + (size_t)units * 4, st) != cudaSuccess) return PTENC_ECUDA;
   // the same choice of instantiation as ptenc_decode_attn makes for a call over all layers
   const bool lng = use_long_variant(*cfg, cfg->n_layers, tile_n);

@@ -41,6 +41,7 @@ struct PtencDev {
   int* tickets;                 // [L][B][Hkv] arrival counters, self-cleaning
   int part_slots;
   int* status;
+  int* work;                    // next work item of the running attention launch; zero between launches
   // ---- importance-aware eviction (policy PTENC_POLICY_SCORE); all null / zero under the sliding-window policy -------
   int policy, recent;
   int wb;                       // 32-bit words of one sequence's liveness bitmap

@@ -98,7 +98,7 @@ k_append_evict(PtencDev p, int l0, const char* __restrict__ k_new, const char* _
 __global__ void k_reset(PtencDev p, const uint8_t* __restrict__ mask, int clear_status) {
   const int l = blockIdx.x / p.B;
   const int b = blockIdx.x - l * p.B;
-  if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
+  if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) { *p.status = 0; *p.work = 0; }
   if (mask != nullptr && mask[b] == 0) return;
   const long long lb = (long long)l * p.B + b;
   if (threadIdx.x == 0) {
