@@ -356,24 +356,107 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
 
   if (warp == NW) {
     // ================================================================ producer warp
-    // All lanes look an item up (ballots and scans over the chunk prefixes); lane 0 owns the barriers and issues.
-    uint32_t kw[NW];                                         // tiles issued so far for each consumer warp
-#pragma unroll
-    for (int w = 0; w < NW; ++w) kw[w] = 0;
+    // All lanes look an item up (ballots and scans over the chunk prefixes); lane 0 posts the item's description and
+    // its Q rows; lane w < NW feeds consumer warp w: it issues the tiles i = w (mod NW) of every item into that warp's
+    // stages.  One lane issuing every tile of the CTA (a barrier wait, the transaction count and four bulk copies
+    // per tile, ~0.3 us) could just keep up with one SM's share of the HBM stream and fell behind at every item
+    // boundary; NW lanes in parallel have headroom.
+    uint32_t kmine = 0;                                      // tiles this lane has issued into its warp's stages
     uint32_t useq = 0;                                       // items handed to the consumers
     bool aborted = false;
     const long long rows_total = (long long)p.L * B * Hkv * W;
+
+    // Looking an item up (which entry, head and piece it is) needs the ring words of up to 32 entries, and with
+    // nearly all of the SM's memory used as shared memory those loads miss L1: a round trip through L2 that takes
+    // microseconds under the K/V stream.  So the look-up is split: `begin` finds the chunk of entries and requests
+    // their ring words, `finish` uses them -- and between the two the tiles of the item before are issued.  The
+    // number of an item is requested from the global counter one step earlier still.
+    struct Item { int kind, e, h, k, iu_lo, n_mine, P, slot_base; Entry en; };     // kind 0 bad, 1 item, 2 none left
+    struct Pending { int item, tch, ce_lo, ce_hi; Raw raw; };
+    auto lookup_begin = [&](int item) -> Pending {
+      Pending pd;
+      pd.item = item; pd.tch = -1; pd.ce_lo = pd.ce_hi = 0;
+      pd.raw.head = pd.raw.count = pd.raw.sink = pd.raw.act = 0; pd.raw.n = 0;
+      if (item >= n_items) return pd;
+      for (int base = 0; base < NTHREADS; base += 32) {
+        const int idx = base + lane;
+        const bool hit = idx < NTHREADS && s_items[idx] <= item && item < s_items[idx + 1];
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m != 0) { pd.tch = base + __ffs(m) - 1; break; }
+      }
+      if (pd.tch >= 0) {
+        pd.ce_lo = min(pd.tch * chunk, n_ent);
+        pd.ce_hi = min(pd.ce_lo + chunk, n_ent);
+        pd.raw = fetch(pd.ce_lo + lane);                     // the first 32 entries of the chunk; clamped, unconditional
+      }
+      return pd;
+    };
+    auto lookup_finish = [&](const Pending& pd) -> Item {
+      Item it;
+      it.kind = 0; it.e = -1; it.h = it.k = it.iu_lo = it.n_mine = it.P = it.slot_base = 0;
+      it.en.head = it.en.count = it.en.sink = it.en.nt = it.en.t0 = it.en.len2 = 0;
+      if (pd.item >= n_items) { it.kind = 2; return it; }
+      if (pd.tch < 0) return it;
+      int rem = pd.item - s_items[pd.tch];
+      int split_before = s_split[pd.tch];
+      for (int base = pd.ce_lo; base < pd.ce_hi && it.e < 0; base += 32) {
+        const int ee = base + lane;
+        const Entry le = (ee >= pd.ce_hi) ? make_entry(pd.raw, -1)
+                                          : (base == pd.ce_lo ? make_entry(pd.raw, ee) : load_entry(ee));
+        const int pc = pieces_of(le.nt);
+        const int cnt = Hkv * pc, sp = pc > 1 ? cnt : 0;
+        int c_inc = cnt, s_inc = sp;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int a = __shfl_up_sync(0xffffffffu, c_inc, o), c = __shfl_up_sync(0xffffffffu, s_inc, o);
+          if (lane >= o) { c_inc += a; s_inc += c; }
+        }
+        const bool hit = cnt > 0 && c_inc - cnt <= rem && rem < c_inc;
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m != 0) {
+          const int src = __ffs(m) - 1;
+          it.e = base + src;
+          rem -= __shfl_sync(0xffffffffu, c_inc - cnt, src);
+          split_before += __shfl_sync(0xffffffffu, s_inc - sp, src);
+          it.en.head = __shfl_sync(0xffffffffu, le.head, src);
+          it.en.count = __shfl_sync(0xffffffffu, le.count, src);
+          it.en.sink = __shfl_sync(0xffffffffu, le.sink, src);
+          it.en.nt = __shfl_sync(0xffffffffu, le.nt, src);
+          it.en.t0 = __shfl_sync(0xffffffffu, le.t0, src);
+          it.en.len2 = __shfl_sync(0xffffffffu, le.len2, src);
+        } else {
+          rem -= __shfl_sync(0xffffffffu, c_inc, 31);
+          split_before += __shfl_sync(0xffffffffu, s_inc, 31);
+        }
+      }
+      it.P = pieces_of(it.en.nt);
+      if (it.e < 0 || it.P <= 0 || rem < 0 || rem >= Hkv * it.P) return it;
+      it.h = rem / it.P;
+      it.k = rem - it.h * it.P;
+      it.iu_lo = (int)((long long)it.k * it.en.nt / it.P);
+      it.n_mine = (int)((long long)(it.k + 1) * it.en.nt / it.P) - it.iu_lo;
+      it.slot_base = it.P > 1 ? split_before + it.h * it.P : 0;
+      if (it.n_mine <= 0 || it.slot_base + it.P > p.part_slots) return it;
+      it.kind = 1;
+      return it;
+    };
+    auto grab = [&]() -> int { return lane == 0 ? atomicAdd(p.work, 1) : 0; };
+
+    int grabbed = grab();                                    // number of the first item
+    Item cur = lookup_finish(lookup_begin(__shfl_sync(0xffffffffu, grabbed, 0)));
+    if (cur.kind == 1) grabbed = grab();                     // every CTA makes exactly one grab that finds nothing left
     while (!aborted) {
-      int item = 0;
-      if (lane == 0) item = atomicAdd(p.work, 1);
-      item = __shfl_sync(0xffffffffu, item, 0);
       const uint32_t ubuf = useq & 1;
       volatile int* dsc = desc + ubuf * 16;
-      if (item >= n_items) {
-        // nothing left: tell the consumers, and the CTA that makes the very last grab of the launch rewinds the
-        // counter for the next one
+      if (cur.kind != 1) {
+        if (cur.kind == 0) {                                 // uniform over the warp
+          if (lane == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
+          aborted = true;
+          break;
+        }
+        // nothing left: tell the consumers, and the CTA whose grab was the very last of the launch rewinds the counter
         if (lane == 0) {
-          if (item == n_items + (int)gridDim.x - 1) *p.work = 0;
+          if (grabbed == n_items + (int)gridDim.x - 1) *p.work = 0;
           if (mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) {
             dsc[0] = 2;
             mbar_arrive(bar_qfull + 8 * ubuf);
@@ -383,119 +466,64 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         }
         break;
       }
-      // ---- which (entry, head, piece) is item number `item` --------------------------------------------------
-      int tch = -1;
-      for (int base = 0; base < NTHREADS; base += 32) {
-        const int idx = base + lane;
-        const bool hit = idx < NTHREADS && s_items[idx] <= item && item < s_items[idx + 1];
-        const unsigned m = __ballot_sync(0xffffffffu, hit);
-        if (m != 0) { tch = base + __ffs(m) - 1; break; }
-      }
-      Entry en;
-      en.head = en.count = en.sink = en.nt = en.t0 = en.len2 = 0;
-      int e = -1, rem = 0, split_before = 0;
-      if (tch >= 0) {
-        rem = item - s_items[tch];
-        split_before = s_split[tch];
-        const int ce_lo = min(tch * chunk, n_ent), ce_hi = min(ce_lo + chunk, n_ent);
-        for (int base = ce_lo; base < ce_hi && e < 0; base += 32) {
-          const int ee = base + lane;
-          Entry le = load_entry(ee < ce_hi ? ee : -1);
-          const int pc = pieces_of(le.nt);
-          const int it = Hkv * pc, sp = pc > 1 ? it : 0;
-          int it_inc = it, sp_inc = sp;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const int a = __shfl_up_sync(0xffffffffu, it_inc, o), c = __shfl_up_sync(0xffffffffu, sp_inc, o);
-            if (lane >= o) { it_inc += a; sp_inc += c; }
-          }
-          const bool hit = it > 0 && it_inc - it <= rem && rem < it_inc;
-          const unsigned m = __ballot_sync(0xffffffffu, hit);
-          if (m != 0) {
-            const int src = __ffs(m) - 1;
-            e = base + src;
-            rem -= __shfl_sync(0xffffffffu, it_inc - it, src);
-            split_before += __shfl_sync(0xffffffffu, sp_inc - sp, src);
-            en.head = __shfl_sync(0xffffffffu, le.head, src);
-            en.count = __shfl_sync(0xffffffffu, le.count, src);
-            en.sink = __shfl_sync(0xffffffffu, le.sink, src);
-            en.nt = __shfl_sync(0xffffffffu, le.nt, src);
-            en.t0 = __shfl_sync(0xffffffffu, le.t0, src);
-            en.len2 = __shfl_sync(0xffffffffu, le.len2, src);
-          } else {
-            rem -= __shfl_sync(0xffffffffu, it_inc, 31);
-            split_before += __shfl_sync(0xffffffffu, sp_inc, 31);
-          }
-        }
-      }
-      const int P = pieces_of(en.nt);
-      if (e < 0 || P <= 0 || rem < 0 || rem >= Hkv * P) {      // uniform over the warp
-        if (lane == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
-        aborted = true;
-        break;
-      }
-      const int h = rem / P, k = rem - h * P;
-      const int iu_lo = (int)((long long)k * en.nt / P), iu_hi = (int)((long long)(k + 1) * en.nt / P);
-      const int n_mine = iu_hi - iu_lo;
-      const int slot_base = P > 1 ? split_before + h * P : 0;
-      if (n_mine <= 0 || slot_base + P > p.part_slots) {
-        if (lane == 0) atomicOr(p.status, PTENC_ST_BAD_SCHEDULE);
-        aborted = true;
-        break;
-      }
+      const int e = cur.e, h = cur.h, n_mine = cur.n_mine, iu_lo = cur.iu_lo;
+      const Entry en = cur.en;
+      const int li = e / B, b = e - li * B;
       if (lane == 0) {
-        const int li = e / B, b = e - li * B;
-        const size_t lb = (size_t)(l0 + li) * B + b;
         // the item's description and the Q rows of its unit
         if (!mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) { aborted = true; }
         if (!aborted) {
           dsc[1] = li; dsc[2] = b; dsc[3] = h; dsc[4] = en.head; dsc[5] = en.count; dsc[6] = en.sink;
-          dsc[7] = en.t0; dsc[8] = en.len2; dsc[9] = iu_lo; dsc[10] = n_mine; dsc[11] = P; dsc[12] = k;
-          dsc[13] = slot_base; dsc[0] = 1;
+          dsc[7] = en.t0; dsc[8] = en.len2; dsc[9] = iu_lo; dsc[10] = n_mine; dsc[11] = cur.P; dsc[12] = cur.k;
+          dsc[13] = cur.slot_base; dsc[0] = 1;
           const uint32_t qbytes = (uint32_t)(g * D * 2);
           mbar_expect_tx(bar_qfull + 8 * ubuf, qbytes);
           bulk_load(smem_base + SM::OFF_Q + ubuf * SM::Q_BYTES,
                     q + (((size_t)li * B + b) * p.Hq + (size_t)h * g) * D, qbytes, bar_qfull + 8 * ubuf);
-          const long long row0 = ((long long)lb * Hkv + h) * W;
-          for (int i0 = 0; i0 < n_mine && !aborted; i0 += NW) {
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-              if (i0 + w >= n_mine || aborted) continue;
-              const int iu = iu_lo + i0 + w;                 // tile of the unit, in its enumeration order
-              const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
-              const uint32_t s = w * SPW + kw[w] % SPW;
-              const long long yy = row0 + (long long)j * TILE_N;
-              if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
-                atomicOr(p.status, PTENC_ST_BAD_INDEX); aborted = true; continue;
-              }
-              if (!mbar_wait(bar_empty + 8 * s, ((kw[w] / SPW) & 1) ^ 1)) { aborted = true; continue; }
-              const uint32_t dst = smem_base + s * SM::STAGE_BYTES;
-              const uint32_t fb = bar_full + 8 * s;
-              mbar_expect_tx(fb, SM::STAGE_BYTES);
-              const int y = (int)yy;
-#pragma unroll
-              for (int hf = 0; hf < D / 64; ++hf) {
-                tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
-                tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
-              }
-              kw[w] += 1;
-            }
-          }
         }
       }
+      // the next item: its number has arrived by now; request its entries' ring words, and the number after it
+      const int item2 = __shfl_sync(0xffffffffu, grabbed, 0);
+      const Pending pd = lookup_begin(item2);
+      if (item2 < n_items) grabbed = grab();
       aborted = __shfl_sync(0xffffffffu, aborted ? 1 : 0, 0) != 0;
+      if (lane < NW && !aborted) {
+        const size_t lb = (size_t)(l0 + li) * B + b;
+        const long long row0 = ((long long)lb * Hkv + h) * W;
+        for (int i = lane; i < n_mine; i += NW) {
+          const int iu = iu_lo + i;                          // tile of the unit, in its enumeration order
+          const int j = iu < en.len2 ? en.t0 + iu : iu - en.len2;
+          const uint32_t s = lane * SPW + kmine % SPW;
+          const long long yy = row0 + (long long)j * TILE_N;
+          if (j < 0 || j >= n_t || yy < 0 || yy >= rows_total) {
+            atomicOr(p.status, PTENC_ST_BAD_INDEX); aborted = true; break;
+          }
+          if (!mbar_wait(bar_empty + 8 * s, ((kmine / SPW) & 1) ^ 1)) { aborted = true; break; }
+          const uint32_t dst = smem_base + s * SM::STAGE_BYTES;
+          const uint32_t fb = bar_full + 8 * s;
+          mbar_expect_tx(fb, SM::STAGE_BYTES);
+          const int y = (int)yy;
+#pragma unroll
+          for (int hf = 0; hf < D / 64; ++hf) {
+            tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
+            tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
+          }
+          kmine += 1;
+        }
+      }
+      aborted = __any_sync(0xffffffffu, aborted);
+      cur = lookup_finish(pd);
       ++useq;
     }
-    if (lane == 0 && aborted) {
-      atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT);
-      misc[0] = 1;
+    aborted = __any_sync(0xffffffffu, aborted);
+    if (aborted) {
+      if (lane == 0) { atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT); misc[0] = 1; }
       // copies still in flight must land before the CTA's shared memory goes away
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        const uint32_t back = kw[w] < (uint32_t)SPW ? kw[w] : (uint32_t)SPW;
+      if (lane < NW) {
+        const uint32_t back = kmine < (uint32_t)SPW ? kmine : (uint32_t)SPW;
         for (uint32_t i = 0; i < back; ++i) {
-          const uint32_t kk = kw[w] - 1 - i;
-          (void)mbar_wait(bar_full + 8 * (w * SPW + kk % SPW), (kk / SPW) & 1);
+          const uint32_t kk = kmine - 1 - i;
+          (void)mbar_wait(bar_full + 8 * (lane * SPW + kk % SPW), (kk / SPW) & 1);
         }
       }
     }
