@@ -83,8 +83,8 @@ typedef struct {
   int32_t normalize_mode;  /* PTENC_NORM_*                                                          */
   int32_t encode_enabled;  /* 0: state stays at its initial value ("Global-Only" ablation, Sec. 4.3) */
   int32_t device;          /* CUDA device ordinal the workspace lives on                            */
-  int32_t attn_consumer_warps; /* tuning knob of the bf16 tensor-core attention kernel: 0 = chosen per launch
-                                  (three warps on long launches of long windows, four otherwise), 3 or 4 = fixed  */
+  int32_t attn_consumer_warps; /* tuning knob of the bf16 tensor-core attention kernel: warps that consume K/V
+                                  tiles, 0 = the default (four), 3 or 4 = that many                               */
   int32_t policy;          /* PTENC_POLICY_*: which tokens leave when the cache is full                       */
   int32_t recent;          /* PTENC_POLICY_SCORE only: the newest `recent` tokens are never evicted (0..W-1);
                               must be 0 under PTENC_POLICY_FIFO                                               */
@@ -245,10 +245,9 @@ PTENC_API int ptenc_cache_info(ptenc_cache* c, int32_t* tensor_core_attn /*host,
                                int32_t* attn_grid /*host, out*/, int32_t* tensor_core_encode /*host, out*/);
 
 /* What the next attention launch through this handle would run for `layer` (-1 = all layers in one call), host only,
- * every output nullable: *consumer_warps = warps that consume K/V tiles in the tensor-core kernel (3 or 4; chosen
- * per launch from the tiles the call can hold unless ptenc_config.attn_consumer_warps fixes it), *tile_tokens =
- * tokens per K/V tile, *stages = shared-memory pipeline stages.  All three are 0 when the shape-generic kernel
- * serves the cache. */
+ * every output nullable: *consumer_warps = warps that consume K/V tiles in the tensor-core kernel (4 unless
+ * ptenc_config.attn_consumer_warps says 3), *tile_tokens = tokens per K/V tile, *stages = shared-memory pipeline
+ * stages.  All three are 0 when the shape-generic kernel serves the cache. */
 PTENC_API int ptenc_attn_launch_info(ptenc_cache* c, int layer, int32_t* consumer_warps /*host, out*/,
                                      int32_t* tile_tokens /*host, out*/, int32_t* stages /*host, out*/);
 

@@ -902,29 +902,18 @@ template <int D> struct Pick {
   static constexpr int TILE_N = (D == 128) ? PTENC_ATTN_TILE_N_128 : 64;
   static constexpr int STAGES = (D == 128) ? PTENC_ATTN_STAGES_128 : 12;
 };
-// Long launches run under the power cap, and there three consumer warps sustain 2-3 % more bandwidth than four
-// (measured medians of 500+ back-to-back launches: 7B shape 6947 vs 6820 GB/s, Llama shape 7156 vs 6926, 4096-token
-// windows 7060 vs 6858); short launches and short windows (few tiles per unit, more merging per byte) are better off
-// with four (3B shape 6318 vs 6470, 512-token windows 6100 vs 6365).  The choice is made per launch from the
-// number of tiles the call can hold.
+// Two instantiations per head size: four consumer warps (the default) and three.  With one lane issuing all tiles
+// three warps used to sustain a little more bandwidth under the power cap on long launches; since every consumer warp
+// has its own issuing lane four are as fast or faster at every shape measured (7B shape, 1500 back-to-back steps:
+// 2.130 vs 2.147 ms; 512-token windows: 1.156 vs 1.220 ms), so the library no longer switches by itself.  The
+// three-warp instantiation stays selectable through ptenc_config.attn_consumer_warps.
 #ifndef PTENC_ATTN_NW_LONG
 #define PTENC_ATTN_NW_LONG 3
 #endif
-#ifndef PTENC_ATTN_LONG_MIN_TILES_PER_UNIT
-#define PTENC_ATTN_LONG_MIN_TILES_PER_UNIT 32
-#endif
-#ifndef PTENC_ATTN_LONG_MIN_TILES
-#define PTENC_ATTN_LONG_MIN_TILES 300000
-#endif
 constexpr int NW_LONG = PTENC_ATTN_NW_LONG;
 inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
-  // ptenc_config.attn_consumer_warps fixes the choice when it names one of the two instantiations
-  if (cfg.attn_consumer_warps == NW_LONG) return true;
-  if (cfg.attn_consumer_warps == NW_DEFAULT) return false;
-  if (NW_DEFAULT != 4) return false;                    // only when the default was not overridden at build time
-  const long long n_t = (cfg.window + tile_n - 1) / tile_n;
-  const long long tiles = (long long)nl * cfg.batch * cfg.n_kv_heads * n_t;
-  return n_t >= PTENC_ATTN_LONG_MIN_TILES_PER_UNIT && tiles >= PTENC_ATTN_LONG_MIN_TILES;
+  (void)nl; (void)tile_n;
+  return cfg.attn_consumer_warps == NW_LONG && NW_LONG != NW_DEFAULT;
 }
 
 template <int D, int NW, bool SCORE>

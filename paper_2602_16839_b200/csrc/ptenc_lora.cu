@@ -180,23 +180,44 @@ __host__ __device__ inline int lm_k_split(int r) {
   const int tiles = r >> 3;
   return tiles < LM_WARPS ? LM_WARPS / tiles : 1;
 }
-__host__ __device__ inline size_t lr_mma_smem(int G, int r) {
-  // u partials [KS][16][r] fp32 | u of this CTA [16][r] fp32 | w_hi, w_lo [16][G] bf16
-  return (size_t)(lm_k_split(r) + 1) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
+// Shared memory of a CTA: a staging buffer (first the CTA's column slice of the 16 input rows and of B's r rows,
+// later its slice of A's rows), then u partials [KS][16][r] fp32, u of this CTA [16][r] fp32, w_hi and w_lo [16][G] bf16.
+__host__ __device__ inline int lm_slice_pairs(int d_in) { return ((d_in >> 5) + LM_CLUSTER - 1) / LM_CLUSTER; }
+__host__ __device__ inline int lm_row_stride(int d_in) { return lm_slice_pairs(d_in) * 64 + 64; }   // bytes; 64 mod 128
+__host__ __device__ inline size_t lm_stage_bytes(int G, int r, int d_in, int d_out) {
+  const size_t in_bytes = (size_t)(LM_SEQ + r) * lm_row_stride(d_in);
+  const size_t a_rows = (size_t)(((d_out >> 3) + LM_CLUSTER - 1) / LM_CLUSTER) * 8;
+  const size_t a_bytes = a_rows * G * 2;
+  return ((in_bytes > a_bytes ? in_bytes : a_bytes) + 127) & ~(size_t)127;
+}
+__host__ __device__ inline size_t lr_mma_smem(int G, int r, int d_in, int d_out) {
+  return lm_stage_bytes(G, r, d_in, d_out) + (size_t)(lm_k_split(r) + 1) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
 }
 
-// grid = (LM_CLUSTER, nl * ceil(B / 16)), cluster = (LM_CLUSTER, 1, 1)
-__global__ void __cluster_dims__(LM_CLUSTER, 1, 1) __launch_bounds__(LM_THREADS)
+__device__ __forceinline__ void lm_cp16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+__device__ __forceinline__ void lm_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void lm_cp_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// grid = (LM_CLUSTER, nl * ceil(B / 16)), cluster = (LM_CLUSTER, 1, 1).
+// Every global read of a CTA is requested up front or as early as its buffer is free, so that a CTA pays about two
+// memory round trips in all: the column slices of the inputs and of B go to shared memory with asynchronous copies,
+// the state rows and the old outputs go to registers, and the CTA's rows of A follow into the same buffer as soon as
+// the first product is done (while the partial sums travel through the cluster).
+__global__ void __cluster_dims__(LM_CLUSTER, 1, 1) __launch_bounds__(LM_THREADS, 2)
 k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ Bm,
                      const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                      const uint8_t* __restrict__ active, int d_in, int d_out) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ __align__(16) uint8_t lm_smem[];
+  extern __shared__ __align__(128) uint8_t lm_smem[];
   const int G = p.G, r = p.r, B = p.B;
   const int n_tiles = r >> 3;                                   // column tiles of u
   const int KS = lm_k_split(r);                                 // warps sharing a tile split the CTA's slice of d_in
-  float* u_part = reinterpret_cast<float*>(lm_smem);            // [KS][16][r]
+  uint8_t* stage = lm_smem;
+  float* u_part = reinterpret_cast<float*>(lm_smem + lm_stage_bytes(G, r, d_in, d_out));   // [KS][16][r]
   float* u_loc = u_part + KS * LM_SEQ * r;                      // [16][r] this CTA's share of the contraction
   __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u_loc + LM_SEQ * r);    // [16][G]
   __nv_bfloat16* w_lo = w_hi + LM_SEQ * G;
@@ -218,54 +239,65 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
   // this CTA's shares: pairs of mma steps along d_in, tiles of 8 outputs along d_out, sequences of the block
   const int n_pairs = d_in >> 5;
   const int p_lo = rank * n_pairs / LM_CLUSTER, p_hi = (rank + 1) * n_pairs / LM_CLUSTER;
+  const int np = p_hi - p_lo;
   const int n_out_tiles = d_out >> 3;
   const int t_lo = rank * n_out_tiles / LM_CLUSTER, t_hi = (rank + 1) * n_out_tiles / LM_CLUSTER;
   const int s_first = rank * (LM_SEQ / LM_CLUSTER);
+  const int rs = lm_row_stride(d_in);                           // bytes between staged rows
 
-  // ---- what the later phases read is asked into L2 now (128-byte lines) -------------------------------------------------
+  // ---- requests: input and B column slices -> shared memory (rows 0..15 inputs, 16.. B) ---------------------------------
   {
-    const char* pS = reinterpret_cast<const char*>(p.S + ((size_t)l * B + b0 + s_first) * G * r);
-    const int ns4 = max(0, min(LM_SEQ / LM_CLUSTER, nseq - s_first));
-    for (size_t o = (size_t)tid * 128; o < (size_t)ns4 * G * r * 4; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(pS + o));
-    const char* pA = reinterpret_cast<const char*>(Al + (size_t)t_lo * 8 * G);
-    for (size_t o = (size_t)tid * 128; o < (size_t)(t_hi - t_lo) * 8 * G * 2; o += (size_t)LM_THREADS * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(pA + o));
-    for (int s = 0; s < nseq; ++s) {
-      const char* py = reinterpret_cast<const char*>(yl + (size_t)s * d_out + (size_t)t_lo * 8);
-      for (size_t o = (size_t)tid * 128; o < (size_t)(t_hi - t_lo) * 16; o += (size_t)LM_THREADS * 128)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(py + o));
+    const int vec_per_row = np * 4;                             // 16-byte vectors of a row's slice
+    const int rows = LM_SEQ + r;
+    for (int idx = tid; idx < rows * vec_per_row; idx += LM_THREADS) {
+      const int row = idx / vec_per_row, v = idx - row * vec_per_row;
+      uint8_t* dst = stage + (size_t)row * rs + v * 16;
+      if (row < LM_SEQ) {
+        if (row < nseq) lm_cp16(dst, xl + (size_t)row * d_in + (size_t)p_lo * 32 + v * 8);
+        else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+      } else {
+        lm_cp16(dst, Bl + (size_t)(row - LM_SEQ) * d_in + (size_t)p_lo * 32 + v * 8);
+      }
+    }
+    lm_cp_commit();
+  }
+  // ---- requests: the state rows this thread needs in phase 2 (a warp per sequence, a lane per state row; r <= 32 * 4) -----
+  // and the old outputs of this lane's positions in the CTA's output tiles (phase 3) -> registers
+  const int sq = warp;                                          // sequence of this CTA's four handled by this warp
+  const bool s_warp = sq < LM_SEQ / LM_CLUSTER && s_first + sq < nseq;
+  const bool wr_lo = lo_ok && (active == nullptr || active[b0 + qrow] != 0);
+  const bool wr_hi = hi_ok && (active == nullptr || active[b0 + qrow + 8] != 0);
+  constexpr int YT = 4;                                         // output tiles per warp whose old values are prefetched
+  uint32_t y_lo[YT], y_hi[YT];
+#pragma unroll
+  for (int q = 0; q < YT; ++q) {
+    const int t = t_lo + warp + q * LM_WARPS;                   // tiles t_lo + warp, + 8, + 16, + 24
+    y_lo[q] = y_hi[q] = 0u;
+    if (t < t_hi) {
+      const int i0 = t * 8;
+      if (wr_lo) y_lo[q] = *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol);
+      if (wr_hi) y_hi[q] = *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol);
     }
   }
+  lm_cp_wait_all();
+  __syncthreads();
 
-  // ---- phase 1: u (this CTA's slice of d_in) ------------------------------------------------------------------------------
+  // ---- phase 1: u (this CTA's slice of d_in), fragments from shared memory ------------------------------------------------
   {
-    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-    const int np = p_hi - p_lo;
     for (int item = warp; item < n_tiles * KS; item += LM_WARPS) {
       const int tile = item % n_tiles, ks = item / n_tiles;
-      const int s_lo = p_lo + ks * np / KS, s_hi = p_lo + (ks + 1) * np / KS;
-      const __nv_bfloat16* wrow = Bl + (size_t)(tile * 8 + qrow) * d_in + qcol * 8;
-      const __nv_bfloat16* xlo = xl + (size_t)qrow * d_in + qcol * 8;
-      const __nv_bfloat16* xhi = xlo + (size_t)8 * d_in;
+      const int s_lo = ks * np / KS, s_hi = (ks + 1) * np / KS;
+      const uint8_t* wrow = stage + (size_t)(LM_SEQ + tile * 8 + qrow) * rs + qcol * 16;
+      const uint8_t* xlo = stage + (size_t)qrow * rs + qcol * 16;
+      const uint8_t* xhi = xlo + (size_t)8 * rs;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int s0 = s_lo; s0 < s_hi; s0 += 4) {
-        uint4 bw[4], al[4], ah[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if (s0 + q < s_hi) {
-            bw[q] = __ldg(reinterpret_cast<const uint4*>(wrow + (size_t)(s0 + q) * 32));
-            al[q] = lo_ok ? __ldg(reinterpret_cast<const uint4*>(xlo + (size_t)(s0 + q) * 32)) : zero4;
-            ah[q] = hi_ok ? __ldg(reinterpret_cast<const uint4*>(xhi + (size_t)(s0 + q) * 32)) : zero4;
-          }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if (s0 + q < s_hi) {
-            lr_mma(c, al[q].x, ah[q].x, al[q].y, ah[q].y, bw[q].x, bw[q].y);
-            lr_mma(c, al[q].z, ah[q].z, al[q].w, ah[q].w, bw[q].z, bw[q].w);
-          }
-        }
+#pragma unroll 4
+      for (int s0 = s_lo; s0 < s_hi; ++s0) {
+        const uint4 bw = *reinterpret_cast<const uint4*>(wrow + s0 * 64);
+        const uint4 al = *reinterpret_cast<const uint4*>(xlo + s0 * 64);
+        const uint4 ah = *reinterpret_cast<const uint4*>(xhi + s0 * 64);
+        lr_mma(c, al.x, ah.x, al.y, ah.y, bw.x, bw.y);
+        lr_mma(c, al.z, ah.z, al.w, ah.w, bw.z, bw.w);
       }
       float* dst = u_part + ((size_t)ks * LM_SEQ + qrow) * r + tile * 8 + 2 * qcol;
       dst[0] = c[0];
@@ -275,6 +307,13 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
     }
   }
   __syncthreads();
+  // the staging buffer is free: this CTA's rows of A follow into it while the partial sums are exchanged
+  {
+    const size_t bytes = (size_t)(t_hi - t_lo) * 8 * G * 2;
+    const char* src = reinterpret_cast<const char*>(Al + (size_t)t_lo * 8 * G);
+    for (size_t o = (size_t)tid * 16; o < bytes; o += (size_t)LM_THREADS * 16) lm_cp16(stage + o, src + o);
+    lm_cp_commit();
+  }
   for (int i = tid; i < LM_SEQ * r; i += LM_THREADS) {
     float t = u_part[i];
     for (int ks = 1; ks < KS; ++ks) t += u_part[(size_t)ks * LM_SEQ * r + i];
@@ -287,11 +326,11 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
     const float* u_rem[LM_CLUSTER];
 #pragma unroll
     for (int c = 0; c < LM_CLUSTER; ++c) u_rem[c] = cluster.map_shared_rank(u_loc, c);
-    for (int sq = warp; sq < LM_SEQ / LM_CLUSTER; sq += LM_WARPS) {
+    if (sq < LM_SEQ / LM_CLUSTER) {
       const int s = s_first + sq;
       for (int g = lane; g < G; g += 32) {
         float acc = 0.f;
-        if (s < nseq) {
+        if (s_warp) {
           const float* Srow = p.S + (((size_t)l * B + b0 + s) * G + g) * r;
           for (int j0 = 0; j0 < r; j0 += 32) {                  // eight 16-byte loads of the state row in flight
             float4 sv[8];
@@ -337,60 +376,56 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
       }
     }
   }
-  cluster.sync();                                              // remote reads done: peers may overwrite or exit
+  lm_cp_wait_all();                                            // this thread's part of the rows of A has landed
+  cluster.sync();                                              // remote reads done (peers may exit); A visible to all warps
 
-  // ---- phase 3: y += w A^T for this CTA's share of the outputs, four column tiles per iteration ---------------------------
+  // ---- phase 3: y += w A^T for this CTA's share of the outputs ---------------------------------------------------------------
   {
     const int kp = G >> 5;                                      // pairs of mma steps along G
-    const bool wr_lo = lo_ok && (active == nullptr || active[b0 + qrow] != 0);
-    const bool wr_hi = hi_ok && (active == nullptr || active[b0 + qrow + 8] != 0);
+    const __nv_bfloat16* As = reinterpret_cast<const __nv_bfloat16*>(stage);     // rows t_lo * 8 .. of A
     // the w fragments of the first 32 state rows do not depend on the output tile
     const uint4 wh_l = *reinterpret_cast<const uint4*>(w_hi + qrow * G + qcol * 8);
     const uint4 wh_h = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + qcol * 8);
     const uint4 wl_l = *reinterpret_cast<const uint4*>(w_lo + qrow * G + qcol * 8);
     const uint4 wl_h = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + qcol * 8);
-    for (int t0 = t_lo + warp * 4; t0 < t_hi; t0 += LM_WARPS * 4) {
-      uint4 aw[4];
-      uint32_t yl4[4], yh4[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (t0 + q < t_hi) {
-          const int i0 = (t0 + q) * 8;
-          aw[q] = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + qcol * 8));
-          yl4[q] = wr_lo ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
-          yh4[q] = wr_hi ? *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) : 0u;
-        }
+    int q = 0;
+    for (int t = t_lo + warp; t < t_hi; t += LM_WARPS, ++q) {
+      const int i0 = t * 8;
+      const __nv_bfloat16* arow = As + (size_t)((t - t_lo) * 8 + qrow) * G + qcol * 8;
+      const uint4 aw = *reinterpret_cast<const uint4*>(arow);
+      uint32_t ylo, yhi;
+      if (q < YT) {                                             // prefetched at the start (register index is static below)
+        ylo = q == 0 ? y_lo[0] : (q == 1 ? y_lo[1] : (q == 2 ? y_lo[2] : y_lo[3]));
+        yhi = q == 0 ? y_hi[0] : (q == 1 ? y_hi[1] : (q == 2 ? y_hi[2] : y_hi[3]));
+      } else {
+        ylo = wr_lo ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
+        yhi = wr_hi ? *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) : 0u;
       }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (t0 + q >= t_hi) break;
-        const int i0 = (t0 + q) * 8;
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw[q].x, aw[q].y);
-        lr_mma(c, wh_l.z, wh_h.z, wh_l.w, wh_h.w, aw[q].z, aw[q].w);
-        lr_mma(c, wl_l.x, wl_h.x, wl_l.y, wl_h.y, aw[q].x, aw[q].y);
-        lr_mma(c, wl_l.z, wl_h.z, wl_l.w, wl_h.w, aw[q].z, aw[q].w);
-        for (int pp = 1; pp < kp; ++pp) {                       // more than 32 state rows
-          const uint4 bw = __ldg(reinterpret_cast<const uint4*>(Al + (size_t)(i0 + qrow) * G + pp * 32 + qcol * 8));
-          const uint4 a_hl = *reinterpret_cast<const uint4*>(w_hi + qrow * G + pp * 32 + qcol * 8);
-          const uint4 a_hh = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + pp * 32 + qcol * 8);
-          const uint4 a_ll = *reinterpret_cast<const uint4*>(w_lo + qrow * G + pp * 32 + qcol * 8);
-          const uint4 a_lh = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + pp * 32 + qcol * 8);
-          lr_mma(c, a_hl.x, a_hh.x, a_hl.y, a_hh.y, bw.x, bw.y);
-          lr_mma(c, a_hl.z, a_hh.z, a_hl.w, a_hh.w, bw.z, bw.w);
-          lr_mma(c, a_ll.x, a_lh.x, a_ll.y, a_lh.y, bw.x, bw.y);
-          lr_mma(c, a_ll.z, a_lh.z, a_ll.w, a_lh.w, bw.z, bw.w);
-        }
-        if (wr_lo) {
-          const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yl4[q]);
-          *reinterpret_cast<uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) =
-              lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
-        }
-        if (wr_hi) {
-          const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yh4[q]);
-          *reinterpret_cast<uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) =
-              lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
-        }
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw.x, aw.y);
+      lr_mma(c, wh_l.z, wh_h.z, wh_l.w, wh_h.w, aw.z, aw.w);
+      lr_mma(c, wl_l.x, wl_h.x, wl_l.y, wl_h.y, aw.x, aw.y);
+      lr_mma(c, wl_l.z, wl_h.z, wl_l.w, wl_h.w, aw.z, aw.w);
+      for (int pp = 1; pp < kp; ++pp) {                         // more than 32 state rows
+        const uint4 bw = *reinterpret_cast<const uint4*>(arow + pp * 32);
+        const uint4 a_hl = *reinterpret_cast<const uint4*>(w_hi + qrow * G + pp * 32 + qcol * 8);
+        const uint4 a_hh = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + pp * 32 + qcol * 8);
+        const uint4 a_ll = *reinterpret_cast<const uint4*>(w_lo + qrow * G + pp * 32 + qcol * 8);
+        const uint4 a_lh = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + pp * 32 + qcol * 8);
+        lr_mma(c, a_hl.x, a_hh.x, a_hl.y, a_hh.y, bw.x, bw.y);
+        lr_mma(c, a_hl.z, a_hh.z, a_hl.w, a_hh.w, bw.z, bw.w);
+        lr_mma(c, a_ll.x, a_lh.x, a_ll.y, a_lh.y, bw.x, bw.y);
+        lr_mma(c, a_ll.z, a_lh.z, a_ll.w, a_lh.w, bw.z, bw.w);
+      }
+      if (wr_lo) {
+        const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&ylo);
+        *reinterpret_cast<uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) =
+            lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
+      }
+      if (wr_hi) {
+        const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yhi);
+        *reinterpret_cast<uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) =
+            lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
       }
     }
   }
@@ -402,12 +437,18 @@ cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* 
                                     void* y, const uint8_t* active, int d_in, int d_out, cudaStream_t st) {
   const PtencDev& p = c->dev;
   // tensor-core path: bf16, r a multiple of 8, G and d_in multiples of 32 (d_in at least 128: a slice per CTA of the
-  // cluster), d_out a multiple of 8
+  // cluster), d_out a multiple of 8, and slices that fit the staging buffer with two CTAs per SM
   if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && d_in >= 128 &&
-      (d_out & 7) == 0 && lr_mma_smem(p.G, p.r) <= 48 * 1024 &&
+      (d_out & 7) == 0 && lr_mma_smem(p.G, p.r, d_in, d_out) <= 100 * 1024 &&
       (long long)nl * ((p.B + LM_SEQ - 1) / LM_SEQ) <= 65535) {
+    const size_t smem = lr_mma_smem(p.G, p.r, d_in, d_out);
+    static bool attr_done_c[PTENC_MAX_DEVICES] = {};
+    if (ptenc_first_use(attr_done_c, c->cfg.device)) {
+      cudaError_t e = cudaFuncSetAttribute(k_lora_apply_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e != cudaSuccess) return e;
+    }
     const int nb = (p.B + LM_SEQ - 1) / LM_SEQ;
-    k_lora_apply_cluster<<<dim3(LM_CLUSTER, nl * nb), LM_THREADS, lr_mma_smem(p.G, p.r), st>>>(
+    k_lora_apply_cluster<<<dim3(LM_CLUSTER, nl * nb), LM_THREADS, smem, st>>>(
         p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, active,
         d_in, d_out);
     c->launches++;

@@ -141,13 +141,13 @@ def test_needle_in_every_tile_small_shapes(warps, W, B):
     assert info["consumer_warps"] == warps and n >= 5 * sum((min(T, W) + 31) // 32 for T in (W - W // 3, W, W + 1))
 
 
-@pytest.mark.parametrize("name", ["qwen7b", "llama8b"])
-def test_needle_in_every_tile_full_size(name):
-    """The launch the benchmark times (all layers, full batch, full window; the library picks three consumer warps
-    here): a needle in every unit at every tile position, for a ring that is not yet full and for one wrapped at an
-    odd slot."""
+@pytest.mark.parametrize("name,warps", [("qwen7b", 0), ("qwen7b", 3), ("llama8b", 0)])
+def test_needle_in_every_tile_full_size(name, warps):
+    """The launch the benchmark times (all layers, full batch, full window): a needle in every unit at every tile
+    position, for a ring that is not yet full and for one wrapped at an odd slot; the 7B shape on both
+    instantiations of the kernel."""
     c = dict(CONFIGS[name])
     W = c["window"]
-    info, n = _run_needles(c, c["n_layers"], [W - 301, W + 1013], 0)
-    assert info["consumer_warps"] == 3
+    info, n = _run_needles(c, c["n_layers"], [W - 301, W + 1013], warps)
+    assert info["consumer_warps"] == (warps or 4)
     assert n >= 2 * (W // 32 - 10) * 5

@@ -49,8 +49,8 @@ def test_tiny_fp32_exhaustive():
     p.close()
 
 
-# storage dtype and, for bf16, the consumer-warp count of the tensor-core attention kernel: 0 = the library's choice
-# (four at these sizes), 3 = the instantiation that long launches of long windows use
+# storage dtype and, for bf16, the consumer-warp count of the tensor-core attention kernel: 0 = the default (four),
+# 3 = the other instantiation
 KERNELS = [("fp32", 0), ("bf16", 0), ("bf16", 3)]
 
 
@@ -556,7 +556,7 @@ def test_reset_clears_stale_split_unit_counters_and_status():
 
 
 def test_launch_info_reports_the_instantiation():
-    """Three consumer warps on long launches of long windows, four otherwise; the configuration can fix either."""
+    """Four consumer warps unless the configuration asks for three."""
     c7 = dict(CONFIGS["qwen7b"])
     kw = dict(n_q_heads=c7["n_q_heads"], n_kv_heads=c7["n_kv_heads"], head_dim=128, dtype="bf16")
     small = pt.Cache(pt.make_config(n_layers=2, batch=2, window=2048, **kw))
@@ -565,11 +565,9 @@ def test_launch_info_reports_the_instantiation():
     forced = pt.Cache(pt.make_config(n_layers=2, batch=2, window=2048, attn_consumer_warps=3, **kw))
     assert forced.attn_launch_info(-1)["consumer_warps"] == 3 and forced.attn_launch_info(0)["consumer_warps"] == 3
     forced.close()
-    full = pt.Cache(pt.make_config(n_layers=28, batch=128, window=2048, **kw))      # the 7B-shaped workload
-    assert full.attn_launch_info(-1)["consumer_warps"] == 3          # 917,504 tiles of 64 per unit
-    assert full.attn_launch_info(0)["consumer_warps"] == 4           # one layer alone is a short launch
-    full.close()
-    torch.cuda.empty_cache()
+    d64 = pt.Cache(pt.make_config(n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, head_dim=64, window=256, dtype="bf16"))
+    assert d64.attn_launch_info(-1) == {"consumer_warps": 4, "tile_tokens": 64, "stages": 12}
+    d64.close()
     gen = pt.Cache(pt.make_config(n_layers=1, batch=2, n_q_heads=4, n_kv_heads=1, head_dim=64, window=64, dtype="fp32"))
     assert gen.attn_launch_info(-1) == {"consumer_warps": 0, "tile_tokens": 0, "stages": 0}
     gen.close()
