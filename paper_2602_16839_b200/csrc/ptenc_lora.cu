@@ -184,10 +184,14 @@ __host__ __device__ inline int lm_k_split(int r) {
 // later its slice of A's rows), then u partials [KS][16][r] fp32, u of this CTA [16][r] fp32, w_hi and w_lo [16][G] bf16.
 __host__ __device__ inline int lm_slice_pairs(int d_in) { return ((d_in >> 5) + LM_CLUSTER - 1) / LM_CLUSTER; }
 __host__ __device__ inline int lm_row_stride(int d_in) { return lm_slice_pairs(d_in) * 64 + 64; }   // bytes; 64 mod 128
+__host__ __device__ inline int lm_slice_tiles(int d_out) { return ((d_out >> 3) + LM_CLUSTER - 1) / LM_CLUSTER; }
+__host__ __device__ inline size_t lm_a_bytes(int G, int d_out) {          // the CTA's rows of A, 128-byte aligned
+  return (((size_t)lm_slice_tiles(d_out) * 8 * G * 2) + 127) & ~(size_t)127;
+}
+__host__ __device__ inline int lm_y_stride(int d_out) { return lm_slice_tiles(d_out) * 16 + 16; }    // bytes
 __host__ __device__ inline size_t lm_stage_bytes(int G, int r, int d_in, int d_out) {
   const size_t in_bytes = (size_t)(LM_SEQ + r) * lm_row_stride(d_in);
-  const size_t a_rows = (size_t)(((d_out >> 3) + LM_CLUSTER - 1) / LM_CLUSTER) * 8;
-  const size_t a_bytes = a_rows * G * 2;
+  const size_t a_bytes = lm_a_bytes(G, d_out) + (size_t)LM_SEQ * lm_y_stride(d_out);
   return ((in_bytes > a_bytes ? in_bytes : a_bytes) + 127) & ~(size_t)127;
 }
 __host__ __device__ inline size_t lr_mma_smem(int G, int r, int d_in, int d_out) {
@@ -249,14 +253,14 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
   {
     const int vec_per_row = np * 4;                             // 16-byte vectors of a row's slice
     const int rows = LM_SEQ + r;
-    for (int idx = tid; idx < rows * vec_per_row; idx += LM_THREADS) {
-      const int row = idx / vec_per_row, v = idx - row * vec_per_row;
-      uint8_t* dst = stage + (size_t)row * rs + v * 16;
-      if (row < LM_SEQ) {
-        if (row < nseq) lm_cp16(dst, xl + (size_t)row * d_in + (size_t)p_lo * 32 + v * 8);
-        else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-      } else {
-        lm_cp16(dst, Bl + (size_t)(row - LM_SEQ) * d_in + (size_t)p_lo * 32 + v * 8);
+    for (int row = warp; row < rows; row += LM_WARPS) {         // a warp per row, a lane per 16 bytes
+      uint8_t* drow = stage + (size_t)row * rs;
+      const __nv_bfloat16* srow = row < LM_SEQ ? xl + (size_t)row * d_in + (size_t)p_lo * 32
+                                               : Bl + (size_t)(row - LM_SEQ) * d_in + (size_t)p_lo * 32;
+      const bool real = row >= LM_SEQ || row < nseq;
+      for (int v = lane; v < vec_per_row; v += 32) {
+        if (real) lm_cp16(drow + v * 16, srow + v * 8);
+        else *reinterpret_cast<uint4*>(drow + v * 16) = make_uint4(0u, 0u, 0u, 0u);
       }
     }
     lm_cp_commit();
@@ -265,20 +269,6 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
   // and the old outputs of this lane's positions in the CTA's output tiles (phase 3) -> registers
   const int sq = warp;                                          // sequence of this CTA's four handled by this warp
   const bool s_warp = sq < LM_SEQ / LM_CLUSTER && s_first + sq < nseq;
-  const bool wr_lo = lo_ok && (active == nullptr || active[b0 + qrow] != 0);
-  const bool wr_hi = hi_ok && (active == nullptr || active[b0 + qrow + 8] != 0);
-  constexpr int YT = 4;                                         // output tiles per warp whose old values are prefetched
-  uint32_t y_lo[YT], y_hi[YT];
-#pragma unroll
-  for (int q = 0; q < YT; ++q) {
-    const int t = t_lo + warp + q * LM_WARPS;                   // tiles t_lo + warp, + 8, + 16, + 24
-    y_lo[q] = y_hi[q] = 0u;
-    if (t < t_hi) {
-      const int i0 = t * 8;
-      if (wr_lo) y_lo[q] = *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol);
-      if (wr_hi) y_hi[q] = *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol);
-    }
-  }
   lm_cp_wait_all();
   __syncthreads();
 
@@ -308,10 +298,16 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
   }
   __syncthreads();
   // the staging buffer is free: this CTA's rows of A follow into it while the partial sums are exchanged
+  uint8_t* ystage = stage + lm_a_bytes(G, d_out);               // [16][ys] the block's old outputs, this CTA's columns
+  const int ys = lm_y_stride(d_out);
   {
     const size_t bytes = (size_t)(t_hi - t_lo) * 8 * G * 2;
     const char* src = reinterpret_cast<const char*>(Al + (size_t)t_lo * 8 * G);
     for (size_t o = (size_t)tid * 16; o < bytes; o += (size_t)LM_THREADS * 16) lm_cp16(stage + o, src + o);
+    const int yv = t_hi - t_lo;                                 // 16-byte vectors (one output tile) per row
+    for (int row = warp; row < nseq; row += LM_WARPS)
+      for (int v = lane; v < yv; v += 32)
+        lm_cp16(ystage + (size_t)row * ys + v * 16, yl + (size_t)row * d_out + (size_t)(t_lo + v) * 8);
     lm_cp_commit();
   }
   for (int i = tid; i < LM_SEQ * r; i += LM_THREADS) {
@@ -388,19 +384,12 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
     const uint4 wh_h = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + qcol * 8);
     const uint4 wl_l = *reinterpret_cast<const uint4*>(w_lo + qrow * G + qcol * 8);
     const uint4 wl_h = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + qcol * 8);
-    int q = 0;
-    for (int t = t_lo + warp; t < t_hi; t += LM_WARPS, ++q) {
-      const int i0 = t * 8;
+    for (int t = t_lo + warp; t < t_hi; t += LM_WARPS) {
       const __nv_bfloat16* arow = As + (size_t)((t - t_lo) * 8 + qrow) * G + qcol * 8;
       const uint4 aw = *reinterpret_cast<const uint4*>(arow);
-      uint32_t ylo, yhi;
-      if (q < YT) {                                             // prefetched at the start (register index is static below)
-        ylo = q == 0 ? y_lo[0] : (q == 1 ? y_lo[1] : (q == 2 ? y_lo[2] : y_lo[3]));
-        yhi = q == 0 ? y_hi[0] : (q == 1 ? y_hi[1] : (q == 2 ? y_hi[2] : y_hi[3]));
-      } else {
-        ylo = wr_lo ? *reinterpret_cast<const uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) : 0u;
-        yhi = wr_hi ? *reinterpret_cast<const uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) : 0u;
-      }
+      uint32_t* py_lo = reinterpret_cast<uint32_t*>(ystage + (size_t)qrow * ys + (t - t_lo) * 16 + qcol * 4);
+      uint32_t* py_hi = reinterpret_cast<uint32_t*>(ystage + (size_t)(qrow + 8) * ys + (t - t_lo) * 16 + qcol * 4);
+      const uint32_t ylo = lo_ok ? *py_lo : 0u, yhi = hi_ok ? *py_hi : 0u;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
       lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw.x, aw.y);
       lr_mma(c, wh_l.z, wh_h.z, wh_l.w, wh_h.w, aw.z, aw.w);
@@ -417,16 +406,23 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
         lr_mma(c, a_ll.x, a_lh.x, a_ll.y, a_lh.y, bw.x, bw.y);
         lr_mma(c, a_ll.z, a_lh.z, a_ll.w, a_lh.w, bw.z, bw.w);
       }
-      if (wr_lo) {
+      if (lo_ok) {
         const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&ylo);
-        *reinterpret_cast<uint32_t*>(yl + (size_t)qrow * d_out + i0 + 2 * qcol) =
-            lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
+        *py_lo = lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
       }
-      if (wr_hi) {
+      if (hi_ok) {
         const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yhi);
-        *reinterpret_cast<uint32_t*>(yl + (size_t)(qrow + 8) * d_out + i0 + 2 * qcol) =
-            lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
+        *py_hi = lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
       }
+    }
+    __syncthreads();
+    // the new outputs leave as whole 16-byte vectors, a warp per row
+    const int yv = t_hi - t_lo;
+    for (int row = warp; row < nseq; row += LM_WARPS) {
+      if (active != nullptr && active[b0 + row] == 0) continue;
+      for (int v = lane; v < yv; v += 32)
+        *reinterpret_cast<uint4*>(yl + (size_t)row * d_out + (size_t)(t_lo + v) * 8) =
+            *reinterpret_cast<const uint4*>(ystage + (size_t)row * ys + v * 16);
     }
   }
 }
