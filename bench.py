@@ -72,7 +72,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes moved (read + written, ncu counters) per algorithmic byte of the tensor-core attention kernel, keyed by
 # window: each ratio was measured on a launch with a smaller batch of the same head shape and window, and DRAM
 # traffic grows in proportion to the K/V tiles a launch reads.  Windows with no capture report no traffic figure.
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2048: 1.0030}
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {512: 1.0132, 2048: 1.0057}
 
 
 def workload_cfg(name: str) -> dict:
@@ -530,7 +530,9 @@ def run_gpu(args, c: dict):
             for i in range(n_done, t + 1):                        # run on to the next evicting step
                 cache.append_evict(-1, pool[i % R][1], pool[i % R][2])
             Ee = min(E, W - P)
+            torch.cuda.nvtx.range_push("ptenc_extras_encode")
             ms = timed(lambda: cache.encode(-1))
+            torch.cuda.nvtx.range_pop()
             by = L * B * (2 * Ee * d_kv * elt + 2 * G * r * 4)
             fl = L * B * Ee * (4 * d_kv * r + 4 * r * r) + L * B * 2 * G * r * r
             extras["encode_burst"] = {"ms": ms, "algorithmic_gbs": by / ms / 1e6, "tflops": fl / ms / 1e9,
@@ -542,7 +544,9 @@ def run_gpu(args, c: dict):
         xin = gen.generic(62, 0, (L, B, d_q), 1.0)
         yio = gen.generic(63, 0, (L, B, d_q), 1.0)
         flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+        torch.cuda.nvtx.range_push("ptenc_extras_lora")
         ms = timed(lambda: cache.lora_apply(-1, Am, Bw, xin, yio), flush=flush)
+        torch.cuda.nvtx.range_pop()
         by = L * (2 * G * d_q * elt + B * (3 * d_q * elt + G * r * 4))
         extras["lora_apply"] = {"ms": ms, "algorithmic_gbs": by / ms / 1e6, "d_in": d_q, "d_out": d_q,
                                 "how": "median of 20 ptenc_lora_apply(layer=-1) calls, L2 flushed, CUDA events"}
@@ -562,7 +566,8 @@ def run_gpu(args, c: dict):
         step_gbs = bm["step"] / (ms_total * 1e-3) / 1e9
         bm["attn"] /= K                                          # per launch / per step averages from here on
         bm["step"] /= K
-        ratio = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(W) if cache_info["tensor_core_attn"] and P == 0 else None
+        counted = cache_info["tensor_core_attn"] and P == 0 and E == 1 and not score_policy   # the captured launch shape
+        ratio = ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(W) if counted else None
         traffic = ratio * bm["attn"] if ratio is not None else None
         bm.pop("attn_per_step")
         line = {

@@ -379,32 +379,52 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
 #pragma unroll
       for (int i = 0; i < KPT; ++i) m2_s[jm * R + k0 + i] = acc[i];
       tc_epi_sync();
-      // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ...
+      // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ...  The old rows are all
+      // requested before the first is used: one memory round trip per unit instead of one per row (with short
+      // chunks, i.e. few tiles per unit, this tail is what bounds the kernel).
       float* S = p.S + ((size_t)l * B + b) * G * R;
+      constexpr int JJ = (R + 31) / 32;
+      constexpr int ROWS = 8;                             // rows of a warp requested together (32 state rows per pass)
       float total = 0.f;
-      for (int gi = ew; gi < G; gi += 4) {
-        float val[(R + 31) / 32];
-        float ss = 0.f;
+      for (int g0 = 0; g0 < G; g0 += 4 * ROWS) {
+        float s_old[ROWS][JJ];
 #pragma unroll
-        for (int jj = 0; jj < (R + 31) / 32; ++jj) {
-          const int k = lane + 32 * jj;
-          val[jj] = 0.f;
-          if (k < R) {
-            float sp = 0.f;
-#pragma unroll 8
-            for (int j = 0; j < R; ++j) sp = fmaf(qa_s[gi * R + j], m2_s[j * R + k], sp);
-            val[jj] = S[gi * R + k] + sp;
-            ss = fmaf(val[jj], val[jj], ss);
+        for (int i = 0; i < ROWS; ++i) {
+          const int gi = g0 + ew + 4 * i;
+#pragma unroll
+          for (int jj = 0; jj < JJ; ++jj) {
+            const int k = lane + 32 * jj;
+            s_old[i][jj] = (gi < G && k < R) ? S[gi * R + k] : 0.f;
           }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        total += ss;
-        const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
+        for (int i = 0; i < ROWS; ++i) {
+          const int gi = g0 + ew + 4 * i;
+          if (gi < G) {                                   // uniform over the warp
+            float val[JJ];
+            float ss = 0.f;
 #pragma unroll
-        for (int jj = 0; jj < (R + 31) / 32; ++jj) {
-          const int k = lane + 32 * jj;
-          if (k < R) S[gi * R + k] = val[jj] * sc;
+            for (int jj = 0; jj < JJ; ++jj) {
+              const int k = lane + 32 * jj;
+              val[jj] = 0.f;
+              if (k < R) {
+                float sp = 0.f;
+#pragma unroll 8
+                for (int j = 0; j < R; ++j) sp = fmaf(qa_s[gi * R + j], m2_s[j * R + k], sp);
+                val[jj] = s_old[i][jj] + sp;
+                ss = fmaf(val[jj], val[jj], ss);
+              }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            total += ss;
+            const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
+#pragma unroll
+            for (int jj = 0; jj < JJ; ++jj) {
+              const int k = lane + 32 * jj;
+              if (k < R) S[gi * R + k] = val[jj] * sc;
+            }
+          }
         }
       }
       if (p.norm_mode == PTENC_NORM_FROBENIUS) {
