@@ -107,6 +107,11 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void tc_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tc_cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tc_epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI) : "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored with the 128-byte swizzle (rows of 128 bytes,
@@ -130,13 +135,16 @@ struct TcSmem {
   static constexpr int A_BYTES = TC_M * TC_KC * 2;                  // 16 KiB (a_rows <= 128 of them are loaded)
   static constexpr int W_BYTES = R * TC_KC * 2;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;
-  static constexpr int OFF_KA = TC_STAGES * STAGE_BYTES;            // fp32 [128][R + 1]
-  static constexpr int OFF_VA = OFF_KA + TC_M * (R + 1) * 4;        // fp32 [128][R] (offset is a multiple of 16)
-  static constexpr int OFF_M2 = OFF_VA + TC_M * R * 4;              // fp32 [R][R]
+  static constexpr int RP = R + 4;                                  // row pitch of k_a / v_a: 16-byte stores of
+                                                                    // consecutive rows fall into distinct banks
+  static constexpr int OFF_KA = TC_STAGES * STAGE_BYTES;            // fp32 [128][RP]
+  static constexpr int OFF_VA = OFF_KA + TC_M * RP * 4;             // fp32 [128][RP], directly behind k_a
+  static constexpr int OFF_M2 = OFF_VA + TC_M * RP * 4;             // fp32 [R][R]
   static constexpr int OFF_BAR = OFF_M2 + R * R * 4;                // mbarriers, TMEM base, flags
-  static constexpr int OFF_QA = OFF_BAR + 128;                      // fp32 [G][R]
-  static size_t total(int G) { return (size_t)OFF_QA + (size_t)G * R * 4 + 1024; }
-  static_assert(OFF_VA % 16 == 0 && STAGE_BYTES % 1024 == 0 && W_BYTES % 1024 == 0, "alignment");
+  static constexpr int OFF_QA = OFF_BAR + 128;                      // fp32 [G][R] Q_a, then [G][R] old state rows
+  static size_t total(int G) { return (size_t)OFF_QA + (size_t)2 * G * R * 4 + 1024; }
+  static_assert(OFF_VA % 16 == 0 && OFF_M2 % 16 == 0 && STAGE_BYTES % 1024 == 0 && W_BYTES % 1024 == 0, "alignment");
+  static_assert(2 * TC_M * RP * 4 >= TC_M * 32 * 4, "the groups' partial sums fit over the row buffers");
 };
 
 struct TcArgs {
@@ -156,8 +164,6 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
                   const TcArgs a) {
   using SM = TcSmem<R>;
   constexpr uint32_t TMEM_COLS = (4 * R < 32) ? 32 : 4 * R;         // two buffers of (k_a | v_a); power of two
-  constexpr int TPJ = TC_EPI / R;                                    // epilogue threads per row j of M2
-  constexpr int KPT = R / TPJ;                                       // columns of M2 per thread
   static_assert(R == 16 || R == 32 || R == 64, "rank");
 
   extern __shared__ uint8_t tc_smem_raw[];
@@ -167,6 +173,7 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
   float* va_s = reinterpret_cast<float*>(smem + SM::OFF_VA);
   float* m2_s = reinterpret_cast<float*>(smem + SM::OFF_M2);
   float* qa_s = reinterpret_cast<float*>(smem + SM::OFF_QA);
+  float* so_s = qa_s + (size_t)p.G * R;
   const uint32_t bar_full = sbase + SM::OFF_BAR;                     // [TC_STAGES]
   const uint32_t bar_empty = bar_full + 8 * TC_STAGES;               // [TC_STAGES]
   const uint32_t bar_tfull = bar_empty + 8 * TC_STAGES;              // [2]
@@ -316,124 +323,191 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
     }
   } else {
     // ================================================================ epilogue: 128 threads, one token row each
+    // M2 += K_a^T V_a runs on 4 x 8 register blocks: SLOTS threads cover the r x r result once, and the 128 threads
+    // form COPIES such groups that each sum the token rows of their own (for r <= 32 a group lies inside one warp
+    // and sums rows that this warp wrote, so a warp barrier orders the exchange).  Every shared-memory value then
+    // feeds four or eight FMAs; one value per FMA made shared-memory bandwidth the bound of the whole kernel.
+    constexpr int RP = SM::RP;
+    constexpr int SLOTS = R * R / 32;
+    constexpr int COPIES = TC_EPI / SLOTS;              // 16, 4, 1 for r = 16, 32, 64
+    constexpr int KG = R / 8;
+    constexpr bool WARP_LOCAL = COPIES >= 4;
     const int et = tid - 64;                            // 0..127
     const int q = warp & 3;                             // TMEM lane quarter this warp may read
     const int row = 32 * q + lane;
-    const int jm = et / TPJ, k0 = (et - jm * TPJ) * KPT;
     const int ew = et >> 5;
+    const int slot = et % SLOTS, copy = et / SLOTS;
+    const int j0 = (slot / KG) * 4, k0 = (slot % KG) * 8;
+    const int rr0 = WARP_LOCAL ? 32 * q + (lane / SLOTS) * SLOTS : 0;
+    float* part = ka_s;                                 // [COPIES][R][R], over the row buffers once they are idle
     uint32_t gt = 0;                                    // 128-token tiles consumed so far
-    int cur_l = -1;
     bool ok = true;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      int l, b;
-      long long row0;
-      const int m = unit(u, &l, &b, &row0);
-      if (m <= 0) continue;                             // uniform over the CTA
-      const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
-      // Q_a of the unit's layer (the previous unit's last reads of it are behind this barrier)
-      tc_epi_sync();
-      if (l != cur_l) {
-        for (int i = et; i < G * R; i += TC_EPI) qa_s[i] = p.Qa[(size_t)l * G * R + i];
-        cur_l = l;
-      }
-      float acc[KPT];
-#pragma unroll
-      for (int i = 0; i < KPT; ++i) acc[i] = 0.f;
-      for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
-        const uint32_t bf = gt & 1;
-        // The four warps must agree on going on: the barriers below count all 128 threads.  Each thread reports its
-        // own wait, thread 0 adds the other roles' flag, and everybody reads the verdict after a barrier.
-        if (!tc_mbar_wait(bar_tfull + 8 * bf, (gt >> 1) & 1, abort_flag)) *epi_abort = 1;
-        if (et == 0 && *abort_flag != 0) *epi_abort = 1;
+    int l = 0, b = 0, m = 0;
+    long long row0 = 0;
+    int u = blockIdx.x;
+    if (u < n_units) m = unit(u, &l, &b, &row0);
+    while (u < n_units && ok) {
+      // the next unit's description is requested now and used after this unit
+      const int u_next = u + (int)gridDim.x;
+      int l_next = 0, b_next = 0, m_next = 0;
+      long long row0_next = 0;
+      if (u_next < n_units) m_next = unit(u_next, &l_next, &b_next, &row0_next);
+      if (m > 0) {                                       // uniform over the CTA
+        const int n_tiles = (m + a.a_rows - 1) / a.a_rows;
+        float* S = p.S + ((size_t)l * B + b) * G * R;
+        // Q_a of the unit's layer and the old state rows travel to shared memory while the tiles are reduced (the
+        // previous unit's last reads of these buffers are behind this barrier)
         tc_epi_sync();
-        if (*epi_abort != 0) { ok = false; break; }
-        tc_fence_after();
-        float kr[R], vr[R];
-        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + bf * 2 * R;
-#pragma unroll
-        for (int c = 0; c < R; c += 16) {
-          tc_ld16(taddr + c, kr + c);
-          tc_ld16(taddr + R + c, vr + c);
+        for (int i = et; i < G * R / 4; i += TC_EPI) {
+          tc_cp_async16(tc_smem_u32(qa_s + 4 * i), p.Qa + (size_t)l * G * R + 4 * i);
+          tc_cp_async16(tc_smem_u32(so_s + 4 * i), S + 4 * i);
         }
-        tc_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * bf);
-        const bool valid = (row < a.a_rows) && (tile * a.a_rows + row < m);
+        tc_cp_async_commit();
+        float acc[4][8];
 #pragma unroll
-        for (int j = 0; j < R; ++j) ka_s[row * (R + 1) + j] = valid ? kr[j] : 0.f;
+        for (int x = 0; x < 4; ++x)
 #pragma unroll
-        for (int j = 0; j < R; j += 4)
-          *reinterpret_cast<float4*>(va_s + row * R + j) =
-              valid ? make_float4(vr[j], vr[j + 1], vr[j + 2], vr[j + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        tc_epi_sync();
-        // M2[jm][k0 .. k0 + KPT) += sum over the tile's rows of k_a[row][jm] * v_a[row][k]
-        for (int rr = 0; rr < TC_M; ++rr) {
-          const float kj = ka_s[rr * (R + 1) + jm];
+          for (int y = 0; y < 8; ++y) acc[x][y] = 0.f;
+        for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
+          const uint32_t bf = gt & 1;
+          // The four warps must agree on going on: the barriers below count all 128 threads.  Each thread reports
+          // its own wait, thread 0 adds the other roles' flag, and everybody reads the verdict after a barrier
+          // (which also orders the previous tile's reads of the row buffers before this tile's writes).
+          if (!tc_mbar_wait(bar_tfull + 8 * bf, (gt >> 1) & 1, abort_flag)) *epi_abort = 1;
+          if (et == 0 && *abort_flag != 0) *epi_abort = 1;
+          tc_epi_sync();
+          if (*epi_abort != 0) { ok = false; break; }
+          tc_fence_after();
+          {
+            float kr[R], vr[R];
+            const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + bf * 2 * R;
 #pragma unroll
-          for (int i = 0; i < KPT; ++i) acc[i] = fmaf(kj, va_s[rr * R + k0 + i], acc[i]);
-        }
-        tc_epi_sync();
-      }
-      if (!ok) break;                                   // uniform: the verdict was read after a barrier
+            for (int c = 0; c < R; c += 16) {
+              tc_ld16(taddr + c, kr + c);
+              tc_ld16(taddr + R + c, vr + c);
+            }
+            tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * bf);
+            const bool valid = (row < a.a_rows) && (tile * a.a_rows + row < m);
+            const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int i = 0; i < KPT; ++i) m2_s[jm * R + k0 + i] = acc[i];
-      tc_epi_sync();
-      // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ...  The old rows are all
-      // requested before the first is used: one memory round trip per unit instead of one per row (with short
-      // chunks, i.e. few tiles per unit, this tail is what bounds the kernel).
-      float* S = p.S + ((size_t)l * B + b) * G * R;
-      constexpr int JJ = (R + 31) / 32;
-      constexpr int ROWS = 8;                             // rows of a warp requested together (32 state rows per pass)
-      float total = 0.f;
-      for (int g0 = 0; g0 < G; g0 += 4 * ROWS) {
-        float s_old[ROWS][JJ];
+            for (int j = 0; j < R; j += 4) {
+              *reinterpret_cast<float4*>(ka_s + row * RP + j) =
+                  valid ? make_float4(kr[j], kr[j + 1], kr[j + 2], kr[j + 3]) : zero;
+              *reinterpret_cast<float4*>(va_s + row * RP + j) =
+                  valid ? make_float4(vr[j], vr[j + 1], vr[j + 2], vr[j + 3]) : zero;
+            }
+          }
+          if (WARP_LOCAL) __syncwarp(); else tc_epi_sync();
+          // acc[x][y] += sum over this group's rows of k_a[row][j0 + x] * v_a[row][k0 + y]
+#pragma unroll 4
+          for (int rr = rr0; rr < rr0 + SLOTS; ++rr) {
+            const float4 k4 = *reinterpret_cast<const float4*>(ka_s + rr * RP + j0);
+            const float4 va = *reinterpret_cast<const float4*>(va_s + rr * RP + k0);
+            const float4 vb = *reinterpret_cast<const float4*>(va_s + rr * RP + k0 + 4);
+            const float kx[4] = {k4.x, k4.y, k4.z, k4.w};
+            const float vy[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
-        for (int i = 0; i < ROWS; ++i) {
-          const int gi = g0 + ew + 4 * i;
+            for (int x = 0; x < 4; ++x)
 #pragma unroll
-          for (int jj = 0; jj < JJ; ++jj) {
-            const int k = lane + 32 * jj;
-            s_old[i][jj] = (gi < G && k < R) ? S[gi * R + k] : 0.f;
+              for (int y = 0; y < 8; ++y) acc[x][y] = fmaf(kx[x], vy[y], acc[x][y]);
           }
         }
+        if (!ok) break;                                 // uniform: the verdict was read after a barrier
+        // the groups' sums meet in shared memory
+        if (COPIES > 1) {
+          tc_epi_sync();                                // every group is done with the row buffers
 #pragma unroll
-        for (int i = 0; i < ROWS; ++i) {
-          const int gi = g0 + ew + 4 * i;
-          if (gi < G) {                                   // uniform over the warp
-            float val[JJ];
-            float ss = 0.f;
+          for (int x = 0; x < 4; ++x) {
+            float* dst = part + (size_t)copy * R * R + (j0 + x) * R + k0;
+            *reinterpret_cast<float4*>(dst) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[x][4], acc[x][5], acc[x][6], acc[x][7]);
+          }
+          tc_epi_sync();
+          for (int o = et; o < R * R / 4; o += TC_EPI) {
+            float4 t = *reinterpret_cast<const float4*>(part + 4 * o);
 #pragma unroll
-            for (int jj = 0; jj < JJ; ++jj) {
-              const int k = lane + 32 * jj;
-              val[jj] = 0.f;
-              if (k < R) {
-                float sp = 0.f;
-#pragma unroll 8
-                for (int j = 0; j < R; ++j) sp = fmaf(qa_s[gi * R + j], m2_s[j * R + k], sp);
-                val[jj] = s_old[i][jj] + sp;
+            for (int c = 1; c < COPIES; ++c) {
+              const float4 w = *reinterpret_cast<const float4*>(part + (size_t)c * R * R + 4 * o);
+              t.x += w.x; t.y += w.y; t.z += w.z; t.w += w.w;
+            }
+            *reinterpret_cast<float4*>(m2_s + 4 * o) = t;
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            float* dst = m2_s + (j0 + x) * R + k0;
+            *reinterpret_cast<float4*>(dst) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[x][4], acc[x][5], acc[x][6], acc[x][7]);
+          }
+        }
+        tc_cp_async_wait_all();
+        tc_epi_sync();                                  // M2, Q_a and the old state rows are in shared memory
+        // S' = Q_a M2, S <- Normalize(S + S'): epilogue warp w takes state rows w, w + 4, ..., eight at a time, a
+        // lane per column
+        constexpr int JJ = (R + 31) / 32;
+        constexpr int ROWS = 8;
+        float total = 0.f;
+        for (int g0 = 0; g0 < G; g0 += 4 * ROWS) {
+          float sp[ROWS][JJ];
+#pragma unroll
+          for (int i = 0; i < ROWS; ++i)
+#pragma unroll
+            for (int jj = 0; jj < JJ; ++jj) sp[i][jj] = 0.f;
+#pragma unroll 2
+          for (int j = 0; j < R; j += 4) {
+            float mm[4][JJ];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+              for (int jj = 0; jj < JJ; ++jj) {
+                const int k = lane + 32 * jj;
+                mm[t][jj] = (k < R) ? m2_s[(j + t) * R + k] : 0.f;
+              }
+#pragma unroll
+            for (int i = 0; i < ROWS; ++i) {
+              const int gi = min(g0 + ew + 4 * i, G - 1);          // rows past G are computed and dropped
+              const float4 q4 = *reinterpret_cast<const float4*>(qa_s + gi * R + j);
+#pragma unroll
+              for (int jj = 0; jj < JJ; ++jj)
+                sp[i][jj] = fmaf(q4.x, mm[0][jj], fmaf(q4.y, mm[1][jj], fmaf(q4.z, mm[2][jj], fmaf(q4.w, mm[3][jj], sp[i][jj]))));
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < ROWS; ++i) {
+            const int gi = g0 + ew + 4 * i;
+            if (gi < G) {                                   // uniform over the warp
+              float val[JJ];
+              float ss = 0.f;
+#pragma unroll
+              for (int jj = 0; jj < JJ; ++jj) {
+                const int k = lane + 32 * jj;
+                val[jj] = (k < R) ? so_s[gi * R + k] + sp[i][jj] : 0.f;
                 ss = fmaf(val[jj], val[jj], ss);
               }
-            }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            total += ss;
-            const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
+              for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+              total += ss;
+              const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
 #pragma unroll
-            for (int jj = 0; jj < JJ; ++jj) {
-              const int k = lane + 32 * jj;
-              if (k < R) S[gi * R + k] = val[jj] * sc;
+              for (int jj = 0; jj < JJ; ++jj) {
+                const int k = lane + 32 * jj;
+                if (k < R) S[gi * R + k] = val[jj] * sc;
+              }
             }
           }
         }
+        if (p.norm_mode == PTENC_NORM_FROBENIUS) {
+          if (lane == 0) frob[ew] = total;
+          tc_epi_sync();
+          const float sc = 1.f / fmaxf(sqrtf(frob[0] + frob[1] + frob[2] + frob[3]), 1e-12f);
+          for (int gi = ew; gi < G; gi += 4)
+            for (int k = lane; k < R; k += 32) S[gi * R + k] *= sc;      // each lane rescales what it stored
+        }
       }
-      if (p.norm_mode == PTENC_NORM_FROBENIUS) {
-        if (lane == 0) frob[ew] = total;
-        tc_epi_sync();
-        const float sc = 1.f / fmaxf(sqrtf(frob[0] + frob[1] + frob[2] + frob[3]), 1e-12f);
-        for (int gi = ew; gi < G; gi += 4)
-          for (int k = lane; k < R; k += 32) S[gi * R + k] *= sc;      // each lane rescales what it stored
-      }
+      u = u_next; l = l_next; b = b_next; m = m_next; row0 = row0_next;
     }
     // after an abort the remaining units are left untouched
     if (!ok && lane == 0) { atomicOr(p.status, PTENC_ST_WAIT_TIMEOUT); *abort_flag = 1; }
