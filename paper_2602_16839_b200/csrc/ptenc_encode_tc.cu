@@ -475,26 +475,33 @@ k_encode_chunk_tc(const PtencDev p, const __grid_constant__ CUtensorMap tmK, con
                 sp[i][jj] = fmaf(q4.x, mm[0][jj], fmaf(q4.y, mm[1][jj], fmaf(q4.z, mm[2][jj], fmaf(q4.w, mm[3][jj], sp[i][jj]))));
             }
           }
+          // the eight rows' sums of squares are reduced side by side (eight shuffles in flight, not a chain of forty)
+          float val[ROWS][JJ], ss[ROWS];
+#pragma unroll
+          for (int i = 0; i < ROWS; ++i) {
+            const int gi = min(g0 + ew + 4 * i, G - 1);
+            ss[i] = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < JJ; ++jj) {
+              const int k = lane + 32 * jj;
+              val[i][jj] = (k < R) ? so_s[gi * R + k] + sp[i][jj] : 0.f;
+              ss[i] = fmaf(val[i][jj], val[i][jj], ss[i]);
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int i = 0; i < ROWS; ++i) ss[i] += __shfl_xor_sync(0xffffffffu, ss[i], o);
 #pragma unroll
           for (int i = 0; i < ROWS; ++i) {
             const int gi = g0 + ew + 4 * i;
             if (gi < G) {                                   // uniform over the warp
-              float val[JJ];
-              float ss = 0.f;
+              total += ss[i];
+              const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss[i]), 1e-12f) : 1.f;
 #pragma unroll
               for (int jj = 0; jj < JJ; ++jj) {
                 const int k = lane + 32 * jj;
-                val[jj] = (k < R) ? so_s[gi * R + k] + sp[i][jj] : 0.f;
-                ss = fmaf(val[jj], val[jj], ss);
-              }
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-              total += ss;
-              const float sc = (p.norm_mode == PTENC_NORM_ROW_L2) ? 1.f / fmaxf(sqrtf(ss), 1e-12f) : 1.f;
-#pragma unroll
-              for (int jj = 0; jj < JJ; ++jj) {
-                const int k = lane + 32 * jj;
-                if (k < R) S[gi * R + k] = val[jj] * sc;
+                if (k < R) S[gi * R + k] = val[i][jj] * sc;
               }
             }
           }
