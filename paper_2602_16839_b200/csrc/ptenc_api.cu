@@ -15,7 +15,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t K, V, head, count, n_app, n_sink, stageK, stageV, n_staged, evict_first, S, S0, Qa, Wk, Wv, enc_set,
-      part_acc, part_ml, tickets, status, total;
+      part_acc, part_ml, tickets, status, lora_u, lora_w, total;
   // importance-aware policy only
   size_t slot_tok, score, live_bits, logits, lse2, pending, fq, fq_head, fq_count, ev_tok, ev_slot;
 };
@@ -77,6 +77,8 @@ Layout make_layout(const ptenc_config* c) {
   o.part_ml = take((size_t)PART_SLOTS * 16 * 4);
   o.tickets = take(L * B * Hkv * 4);
   o.status = take(64);
+  o.lora_u = take((size_t)PTENC_LORA_MAX_PART * L * B * r * 4);     // scratch of the weight update: partial sums of B x
+  o.lora_w = take(2 * L * B * G * 2);                               // and S (B x) as two bf16 terms
   o.slot_tok = o.score = o.live_bits = o.logits = o.lse2 = o.pending = o.fq = o.fq_head = o.fq_count = o.ev_tok =
       o.ev_slot = 0;
   if (c->policy == PTENC_POLICY_SCORE) {
@@ -249,6 +251,8 @@ int ptenc_cache_create(const ptenc_config* cfg, void* ws, size_t bytes, void* st
   d.part_slots = PART_SLOTS;
   d.status = reinterpret_cast<int*>(base + lay.status);
   d.work = d.status + 4;                               // same 64-byte block as the status word
+  c->lora_u = reinterpret_cast<float*>(base + lay.lora_u);
+  c->lora_w = reinterpret_cast<__nv_bfloat16*>(base + lay.lora_w);
   d.policy = cfg->policy; d.recent = cfg->recent; d.wb = 0;
   d.slot_tok = nullptr; d.score = nullptr; d.live_bits = nullptr; d.logits = nullptr; d.lse2 = nullptr;
   d.pending = nullptr; d.fq = nullptr; d.fq_head = nullptr; d.fq_count = nullptr; d.ev_tok = nullptr; d.ev_slot = nullptr;

@@ -58,6 +58,8 @@ struct PtencDev {
   int* ev_slot;                 // [L][B][E] their slots
 };
 
+constexpr int PTENC_LORA_MAX_PART = 16;   // most partial sums of B x per sequence (slices of d_in x parts of a slice)
+
 struct ptenc_cache {
   ptenc_config cfg;
   PtencDev dev;
@@ -81,6 +83,8 @@ struct ptenc_cache {
   CUtensorMap tmWk, tmWv;       // 2-D maps over the encoder weights: rows = L*r, cols = d_kv
   CUtensorMap tmStageK, tmStageV;   // 2-D maps over the staged evicted rows: rows = L*B*E, cols = d_kv
   int tc_stage_box;             // token rows per TMA box of the staged maps
+  float* lora_u;                // [PTENC_LORA_MAX_PART][L][B][r] partial sums of B x (scratch of ptenc_lora_apply)
+  __nv_bfloat16* lora_w;        // [2][L][B][G] S (B x) split into two bf16 terms (scratch of ptenc_lora_apply)
 };
 
 // ---- launchers (each returns a cudaError_t from the launch) -------------------------------------

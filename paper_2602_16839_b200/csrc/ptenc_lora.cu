@@ -4,7 +4,7 @@
 // three thin products per sequence (r x d_in, G x r, d_out x G).  Each sequence has its own state, so this is a
 // batch of tiny products; the only sizeable traffic is A and B, which a CTA reads once for a block of sequences.
 // fp32 accumulation throughout; x, y, A, B in the storage dtype.
-#include <cooperative_groups.h>
+#include <string.h>
 
 #include "ptenc_internal.h"
 
@@ -146,24 +146,32 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// bf16 path: warp-level mma inside a thread-block cluster.  Sixteen sequences are the 16 rows of the A operand; the
-// four CTAs of a cluster share one (layer, block of 16 sequences):
-//   phase 1  u = X B^T     each CTA contracts its quarter of d_in (A fragments straight from the inputs, B fragments
-//                          straight from B, both with one 16-byte load per lane feeding two mma steps; the contraction
-//                          index is permuted the same way on both operands, which leaves the sums unchanged); the
-//                          partial sums meet through distributed shared memory;
-//   phase 2  w = S u       fp32, each CTA for four of the sixteen sequences, a lane per state row; w is split into two
-//                          bf16 terms w_hi + w_lo so that nothing but the final rounding of y is lost; the quarters are
-//                          gathered through distributed shared memory;
-//   phase 3  y += w A^T    each CTA for its quarter of d_out, A's rows as the B operand.
-// Splitting a block four ways makes the call 4 x as many, smaller CTAs: all of them are resident at once (one wave),
-// every weight byte is still read once per 16 sequences, and the three dependent phases of one block overlap with
-// those of the others on the same SM.
+// bf16 path: three streaming kernels on warp-level mma, chained by programmatic dependent launch.  Sixteen sequences
+// are the 16 rows of the A operand of mma.sync.m16n8k16.
+//   k_lora_u   u = X B^T   a CTA per (layer, slice of d_in) keeps its column slice of B in shared memory and streams
+//                          the inputs of every sequence of the layer through registers, a warp per 16 sequences;
+//                          the slices' partial sums go to a scratch area [part][layer][sequence][r];
+//   k_lora_w   w = S u     a warp per (layer, sequence): the partial sums are added in a fixed order, the state is
+//                          read as one coalesced block, w leaves as two bf16 terms w_hi + w_lo so that nothing but
+//                          the final rounding of y is lost;
+//   k_lora_y   y += w A^T  a CTA per (layer, slice of d_out) keeps its rows of A in shared memory and streams the
+//                          old outputs in and the new ones out, 16 bytes per lane and row.
+// Every CTA of the two streaming kernels is resident at once (two per SM); the loads that do not depend on the kernel
+// in front are requested before the wait for it.  (Folding the second product into the third kernel, the CTAs of a
+// layer meeting at a counter, was slower: under load every dependent memory round trip costs about 2.5 us, and that
+// version had more of them in a row.)
+// One 16-byte load per lane feeds two mma steps: the contraction index is permuted the same way on both operands,
+// which leaves the sums unchanged.
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int LM_SEQ = 16;
-constexpr int LM_CLUSTER = 4;
-constexpr int LM_THREADS = 256;
-constexpr int LM_WARPS = LM_THREADS / 32;
+constexpr int LS_THREADS = 256;
+constexpr int LS_WARPS = LS_THREADS / 32;
+#ifndef PTENC_LORA_CB
+#define PTENC_LORA_CB 6
+#endif
+#ifndef PTENC_LORA_CTAS_PER_SM
+#define PTENC_LORA_CTAS_PER_SM 2
+#endif
+constexpr int LS_CB = PTENC_LORA_CB; // 32-wide chunks of the contraction / 32-wide groups of outputs requested together
 
 __device__ __forceinline__ void lr_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -176,255 +184,356 @@ __device__ __forceinline__ uint32_t lr_pack(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__host__ __device__ inline int lm_k_split(int r) {
-  const int tiles = r >> 3;
-  return tiles < LM_WARPS ? LM_WARPS / tiles : 1;
-}
-// Shared memory of a CTA: a staging buffer (first the CTA's column slice of the 16 input rows and of B's r rows,
-// later its slice of A's rows), then u partials [KS][16][r] fp32, u of this CTA [16][r] fp32, w_hi and w_lo [16][G] bf16.
-__host__ __device__ inline int lm_slice_pairs(int d_in) { return ((d_in >> 5) + LM_CLUSTER - 1) / LM_CLUSTER; }
-__host__ __device__ inline int lm_row_stride(int d_in) { return lm_slice_pairs(d_in) * 64 + 64; }   // bytes; 64 mod 128
-__host__ __device__ inline int lm_slice_tiles(int d_out) { return ((d_out >> 3) + LM_CLUSTER - 1) / LM_CLUSTER; }
-__host__ __device__ inline size_t lm_a_bytes(int G, int d_out) {          // the CTA's rows of A, 128-byte aligned
-  return (((size_t)lm_slice_tiles(d_out) * 8 * G * 2) + 127) & ~(size_t)127;
-}
-__host__ __device__ inline int lm_y_stride(int d_out) { return lm_slice_tiles(d_out) * 16 + 16; }    // bytes
-__host__ __device__ inline size_t lm_stage_bytes(int G, int r, int d_in, int d_out) {
-  const size_t in_bytes = (size_t)(LM_SEQ + r) * lm_row_stride(d_in);
-  const size_t a_bytes = lm_a_bytes(G, d_out) + (size_t)LM_SEQ * lm_y_stride(d_out);
-  return ((in_bytes > a_bytes ? in_bytes : a_bytes) + 127) & ~(size_t)127;
-}
-__host__ __device__ inline size_t lr_mma_smem(int G, int r, int d_in, int d_out) {
-  return lm_stage_bytes(G, r, d_in, d_out) + (size_t)(lm_k_split(r) + 1) * LM_SEQ * r * 4 + (size_t)2 * LM_SEQ * G * 2;
-}
-
-__device__ __forceinline__ void lm_cp16(void* smem_dst, const void* gsrc) {
+__device__ __forceinline__ void ls_cp16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
                : "memory");
 }
-__device__ __forceinline__ void lm_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void lm_cp_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void ls_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void ls_cp_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void ls_let_next_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void ls_wait_for_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// grid = (LM_CLUSTER, nl * ceil(B / 16)), cluster = (LM_CLUSTER, 1, 1).
-// Every global read of a CTA is requested up front or as early as its buffer is free, so that a CTA pays about two
-// memory round trips in all: the column slices of the inputs and of B go to shared memory with asynchronous copies,
-// the state rows and the old outputs go to registers, and the CTA's rows of A follow into the same buffer as soon as
-// the first product is done (while the partial sums travel through the cluster).
-__global__ void __cluster_dims__(LM_CLUSTER, 1, 1) __launch_bounds__(LM_THREADS, 2)
-k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ Bm,
-                     const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
-                     const uint8_t* __restrict__ active, int d_in, int d_out) {
-  namespace cg = cooperative_groups;
-  cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ __align__(128) uint8_t lm_smem[];
-  const int G = p.G, r = p.r, B = p.B;
-  const int n_tiles = r >> 3;                                   // column tiles of u
-  const int KS = lm_k_split(r);                                 // warps sharing a tile split the CTA's slice of d_in
-  uint8_t* stage = lm_smem;
-  float* u_part = reinterpret_cast<float*>(lm_smem + lm_stage_bytes(G, r, d_in, d_out));   // [KS][16][r]
-  float* u_loc = u_part + KS * LM_SEQ * r;                      // [16][r] this CTA's share of the contraction
-  __nv_bfloat16* w_hi = reinterpret_cast<__nv_bfloat16*>(u_loc + LM_SEQ * r);    // [16][G]
-  __nv_bfloat16* w_lo = w_hi + LM_SEQ * G;
+// bytes between the staged rows of B: the slice, padded so that the rows of a fragment load fall into distinct banks
+__host__ __device__ inline int ls_b_stride(int np_max) { return (np_max * 64) | 64; }
 
+// grid = (SL, nl).  u_part [SL * KS][nl][B][r] fp32.
+template <int NT>                    // column tiles of u: r = 8 * NT
+__global__ void __launch_bounds__(LS_THREADS, 2)
+k_lora_u(PtencDev p, const __nv_bfloat16* __restrict__ Bm, const __nv_bfloat16* __restrict__ x,
+         float* __restrict__ u_part, int d_in, int SL, int KS) {
+  ls_let_next_start();
+  extern __shared__ __align__(128) uint8_t ls_smem[];
+  constexpr int r = 8 * NT;
+  const int B = p.B, nl = gridDim.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qrow = lane >> 2, qcol = lane & 3;
-  const int rank = (int)cluster.block_rank();                   // = blockIdx.x
-  const int nblk = (B + LM_SEQ - 1) / LM_SEQ;
-  const int li = blockIdx.y / nblk;
-  const int b0 = (blockIdx.y - li * nblk) * LM_SEQ;
-  const int l = l0 + li;
-  const int nseq = min(LM_SEQ, B - b0);
-  const __nv_bfloat16* Bl = Bm + (size_t)li * r * d_in;
-  const __nv_bfloat16* Al = A + (size_t)li * d_out * G;
-  const __nv_bfloat16* xl = x + ((size_t)li * B + b0) * d_in;
-  __nv_bfloat16* yl = y + ((size_t)li * B + b0) * d_out;
-  const bool lo_ok = qrow < nseq, hi_ok = qrow + 8 < nseq;      // the two sequences whose rows this lane touches
-
-  // this CTA's shares: pairs of mma steps along d_in, tiles of 8 outputs along d_out, sequences of the block
+  const int li = blockIdx.y, sl = blockIdx.x;
   const int n_pairs = d_in >> 5;
-  const int p_lo = rank * n_pairs / LM_CLUSTER, p_hi = (rank + 1) * n_pairs / LM_CLUSTER;
-  const int np = p_hi - p_lo;
-  const int n_out_tiles = d_out >> 3;
-  const int t_lo = rank * n_out_tiles / LM_CLUSTER, t_hi = (rank + 1) * n_out_tiles / LM_CLUSTER;
-  const int s_first = rank * (LM_SEQ / LM_CLUSTER);
-  const int rs = lm_row_stride(d_in);                           // bytes between staged rows
+  const int p_lo = sl * n_pairs / SL, np = (sl + 1) * n_pairs / SL - p_lo;
+  const int rs = ls_b_stride((n_pairs + SL - 1) / SL);
+  const __nv_bfloat16* Bl = Bm + (size_t)li * r * d_in + (size_t)p_lo * 32;
+  const __nv_bfloat16* xl = x + (size_t)li * B * d_in + (size_t)p_lo * 32;
 
-  // ---- requests: input and B column slices -> shared memory (rows 0..15 inputs, 16.. B) ---------------------------------
-  {
-    const int vec_per_row = np * 4;                             // 16-byte vectors of a row's slice
-    const int rows = LM_SEQ + r;
-    for (int row = warp; row < rows; row += LM_WARPS) {         // a warp per row, a lane per 16 bytes
-      uint8_t* drow = stage + (size_t)row * rs;
-      const __nv_bfloat16* srow = row < LM_SEQ ? xl + (size_t)row * d_in + (size_t)p_lo * 32
-                                               : Bl + (size_t)(row - LM_SEQ) * d_in + (size_t)p_lo * 32;
-      const bool real = row >= LM_SEQ || row < nseq;
-      for (int v = lane; v < vec_per_row; v += 32) {
-        if (real) lm_cp16(drow + v * 16, srow + v * 8);
-        else *reinterpret_cast<uint4*>(drow + v * 16) = make_uint4(0u, 0u, 0u, 0u);
-      }
+  for (int row = warp; row < r; row += LS_WARPS)               // the slice of B: a warp per row, a lane per 16 bytes
+    for (int v = lane; v < np * 4; v += 32) ls_cp16(ls_smem + (size_t)row * rs + v * 16, Bl + (size_t)row * d_in + v * 8);
+  ls_cp_commit();
+
+  const int n_mt = (B + 15) >> 4;
+  const int n_items = n_mt * KS;                               // (16 sequences, part of the slice) per warp pass
+  uint4 xa[LS_CB], xb[LS_CB];
+  auto request = [&](int item, int c0) {                       // the inputs of up to LS_CB chunks of an item
+    const int mt = item % n_mt, ks = item / n_mt;
+    const int c_hi = (ks + 1) * np / KS;
+    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int i = 0; i < LS_CB; ++i) {
+      const bool in = c0 + i < c_hi;
+      xa[i] = (in && b_lo < B) ? __ldg(reinterpret_cast<const uint4*>(xl + (size_t)b_lo * d_in + (c0 + i) * 32 + qcol * 8)) : zero;
+      xb[i] = (in && b_hi < B) ? __ldg(reinterpret_cast<const uint4*>(xl + (size_t)b_hi * d_in + (c0 + i) * 32 + qcol * 8)) : zero;
     }
-    lm_cp_commit();
-  }
-  // ---- requests: the state rows this thread needs in phase 2 (a warp per sequence, a lane per state row; r <= 32 * 4) -----
-  // and the old outputs of this lane's positions in the CTA's output tiles (phase 3) -> registers
-  const int sq = warp;                                          // sequence of this CTA's four handled by this warp
-  const bool s_warp = sq < LM_SEQ / LM_CLUSTER && s_first + sq < nseq;
-  lm_cp_wait_all();
+  };
+  bool requested = false;
+  if (warp < n_items) { request(warp, (warp / n_mt) * np / KS); requested = true; }   // in flight while B lands
+  ls_cp_wait_all();
   __syncthreads();
 
-  // ---- phase 1: u (this CTA's slice of d_in), fragments from shared memory ------------------------------------------------
-  {
-    for (int item = warp; item < n_tiles * KS; item += LM_WARPS) {
-      const int tile = item % n_tiles, ks = item / n_tiles;
-      const int s_lo = ks * np / KS, s_hi = (ks + 1) * np / KS;
-      const uint8_t* wrow = stage + (size_t)(LM_SEQ + tile * 8 + qrow) * rs + qcol * 16;
-      const uint8_t* xlo = stage + (size_t)qrow * rs + qcol * 16;
-      const uint8_t* xhi = xlo + (size_t)8 * rs;
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-      for (int s0 = s_lo; s0 < s_hi; ++s0) {
-        const uint4 bw = *reinterpret_cast<const uint4*>(wrow + s0 * 64);
-        const uint4 al = *reinterpret_cast<const uint4*>(xlo + s0 * 64);
-        const uint4 ah = *reinterpret_cast<const uint4*>(xhi + s0 * 64);
-        lr_mma(c, al.x, ah.x, al.y, ah.y, bw.x, bw.y);
-        lr_mma(c, al.z, ah.z, al.w, ah.w, bw.z, bw.w);
-      }
-      float* dst = u_part + ((size_t)ks * LM_SEQ + qrow) * r + tile * 8 + 2 * qcol;
-      dst[0] = c[0];
-      dst[1] = c[1];
-      dst[8 * r] = c[2];
-      dst[8 * r + 1] = c[3];
-    }
-  }
-  __syncthreads();
-  // the staging buffer is free: this CTA's rows of A follow into it while the partial sums are exchanged
-  uint8_t* ystage = stage + lm_a_bytes(G, d_out);               // [16][ys] the block's old outputs, this CTA's columns
-  const int ys = lm_y_stride(d_out);
-  {
-    const size_t bytes = (size_t)(t_hi - t_lo) * 8 * G * 2;
-    const char* src = reinterpret_cast<const char*>(Al + (size_t)t_lo * 8 * G);
-    for (size_t o = (size_t)tid * 16; o < bytes; o += (size_t)LM_THREADS * 16) lm_cp16(stage + o, src + o);
-    const int yv = t_hi - t_lo;                                 // 16-byte vectors (one output tile) per row
-    for (int row = warp; row < nseq; row += LM_WARPS)
-      for (int v = lane; v < yv; v += 32)
-        lm_cp16(ystage + (size_t)row * ys + v * 16, yl + (size_t)row * d_out + (size_t)(t_lo + v) * 8);
-    lm_cp_commit();
-  }
-  for (int i = tid; i < LM_SEQ * r; i += LM_THREADS) {
-    float t = u_part[i];
-    for (int ks = 1; ks < KS; ++ks) t += u_part[(size_t)ks * LM_SEQ * r + i];
-    u_loc[i] = t;
-  }
-  cluster.sync();                                              // every CTA's share of u is in its shared memory
-
-  // ---- phase 2: w = S u for this CTA's four sequences (a warp per sequence, a lane per state row) -----------------------
-  {
-    const float* u_rem[LM_CLUSTER];
+  for (int item = warp; item < n_items; item += LS_WARPS) {
+    const int mt = item % n_mt, ks = item / n_mt;
+    const int c_lo = ks * np / KS, c_hi = (ks + 1) * np / KS;
+    float acc[NT][4];
 #pragma unroll
-    for (int c = 0; c < LM_CLUSTER; ++c) u_rem[c] = cluster.map_shared_rank(u_loc, c);
-    if (sq < LM_SEQ / LM_CLUSTER) {
-      const int s = s_first + sq;
-      for (int g = lane; g < G; g += 32) {
-        float acc = 0.f;
-        if (s_warp) {
-          const float* Srow = p.S + (((size_t)l * B + b0 + s) * G + g) * r;
-          for (int j0 = 0; j0 < r; j0 += 32) {                  // eight 16-byte loads of the state row in flight
-            float4 sv[8];
+    for (int t = 0; t < NT; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
+    for (int c0 = c_lo; c0 < c_hi; c0 += LS_CB) {
+      if (!requested) request(item, c0);
+      requested = false;
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              sv[i] = (j0 + 4 * i < r) ? *reinterpret_cast<const float4*>(Srow + j0 + 4 * i)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = 0; i < LS_CB; ++i) {
+        if (c0 + i < c_hi) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int j = j0 + 4 * i;
-              if (j < r) {
-                float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int c = 0; c < LM_CLUSTER; ++c) {           // the same order in every CTA
-                  const float4 t = *reinterpret_cast<const float4*>(u_rem[c] + (size_t)s * r + j);
-                  uu.x += t.x; uu.y += t.y; uu.z += t.z; uu.w += t.w;
-                }
-                acc = fmaf(sv[i].x, uu.x, acc);
-                acc = fmaf(sv[i].y, uu.y, acc);
-                acc = fmaf(sv[i].z, uu.z, acc);
-                acc = fmaf(sv[i].w, uu.w, acc);
-              }
-            }
+          for (int t = 0; t < NT; ++t) {
+            const uint4 bw = *reinterpret_cast<const uint4*>(ls_smem + (size_t)(t * 8 + qrow) * rs + (c0 + i) * 64 + qcol * 16);
+            lr_mma(acc[t], xa[i].x, xb[i].x, xa[i].y, xb[i].y, bw.x, bw.y);
+            lr_mma(acc[t], xa[i].z, xb[i].z, xa[i].w, xb[i].w, bw.z, bw.w);
           }
         }
-        const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-        w_hi[s * G + g] = hi;
-        w_lo[s * G + g] = __float2bfloat16_rn(acc - __bfloat162float(hi));
       }
     }
-  }
-  cluster.sync();                                              // every CTA's four rows of w are in its shared memory
-  // gather the other CTAs' rows of w (16 x G bf16 twice: a few KB)
-  {
-    const int per_cta = (LM_SEQ / LM_CLUSTER) * G;               // elements of w_hi (and of w_lo) a CTA produced
-    for (int c = 0; c < LM_CLUSTER; ++c) {
-      if (c == rank) continue;
-      const __nv_bfloat16* rh = cluster.map_shared_rank(w_hi, c) + c * per_cta;
-      const __nv_bfloat16* rl = cluster.map_shared_rank(w_lo, c) + c * per_cta;
-      for (int i = tid * 8; i < per_cta; i += LM_THREADS * 8) {
-        *reinterpret_cast<uint4*>(w_hi + c * per_cta + i) = *reinterpret_cast<const uint4*>(rh + i);
-        *reinterpret_cast<uint4*>(w_lo + c * per_cta + i) = *reinterpret_cast<const uint4*>(rl + i);
-      }
+    float* dst = u_part + (((size_t)(sl * KS + ks) * nl + li) * B + 16 * mt + qrow) * r + 2 * qcol;
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      if (16 * mt + qrow < B) *reinterpret_cast<float2*>(dst + t * 8) = make_float2(acc[t][0], acc[t][1]);
+      if (16 * mt + qrow + 8 < B) *reinterpret_cast<float2*>(dst + (size_t)8 * r + t * 8) = make_float2(acc[t][2], acc[t][3]);
     }
   }
-  lm_cp_wait_all();                                            // this thread's part of the rows of A has landed
-  cluster.sync();                                              // remote reads done (peers may exit); A visible to all warps
+}
 
-  // ---- phase 3: y += w A^T for this CTA's share of the outputs ---------------------------------------------------------------
-  {
-    const int kp = G >> 5;                                      // pairs of mma steps along G
-    const __nv_bfloat16* As = reinterpret_cast<const __nv_bfloat16*>(stage);     // rows t_lo * 8 .. of A
-    // the w fragments of the first 32 state rows do not depend on the output tile
-    const uint4 wh_l = *reinterpret_cast<const uint4*>(w_hi + qrow * G + qcol * 8);
-    const uint4 wh_h = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + qcol * 8);
-    const uint4 wl_l = *reinterpret_cast<const uint4*>(w_lo + qrow * G + qcol * 8);
-    const uint4 wl_h = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + qcol * 8);
-    for (int t = t_lo + warp; t < t_hi; t += LM_WARPS) {
-      const __nv_bfloat16* arow = As + (size_t)((t - t_lo) * 8 + qrow) * G + qcol * 8;
-      const uint4 aw = *reinterpret_cast<const uint4*>(arow);
-      uint32_t* py_lo = reinterpret_cast<uint32_t*>(ystage + (size_t)qrow * ys + (t - t_lo) * 16 + qcol * 4);
-      uint32_t* py_hi = reinterpret_cast<uint32_t*>(ystage + (size_t)(qrow + 8) * ys + (t - t_lo) * 16 + qcol * 4);
-      const uint32_t ylo = lo_ok ? *py_lo : 0u, yhi = hi_ok ? *py_hi : 0u;
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-      lr_mma(c, wh_l.x, wh_h.x, wh_l.y, wh_h.y, aw.x, aw.y);
-      lr_mma(c, wh_l.z, wh_h.z, wh_l.w, wh_h.w, aw.z, aw.w);
-      lr_mma(c, wl_l.x, wl_h.x, wl_l.y, wl_h.y, aw.x, aw.y);
-      lr_mma(c, wl_l.z, wl_h.z, wl_l.w, wl_h.w, aw.z, aw.w);
-      for (int pp = 1; pp < kp; ++pp) {                         // more than 32 state rows
-        const uint4 bw = *reinterpret_cast<const uint4*>(arow + pp * 32);
-        const uint4 a_hl = *reinterpret_cast<const uint4*>(w_hi + qrow * G + pp * 32 + qcol * 8);
-        const uint4 a_hh = *reinterpret_cast<const uint4*>(w_hi + (qrow + 8) * G + pp * 32 + qcol * 8);
-        const uint4 a_ll = *reinterpret_cast<const uint4*>(w_lo + qrow * G + pp * 32 + qcol * 8);
-        const uint4 a_lh = *reinterpret_cast<const uint4*>(w_lo + (qrow + 8) * G + pp * 32 + qcol * 8);
-        lr_mma(c, a_hl.x, a_hh.x, a_hl.y, a_hh.y, bw.x, bw.y);
-        lr_mma(c, a_hl.z, a_hh.z, a_hl.w, a_hh.w, bw.z, bw.w);
-        lr_mma(c, a_ll.x, a_lh.x, a_ll.y, a_lh.y, bw.x, bw.y);
-        lr_mma(c, a_ll.z, a_lh.z, a_ll.w, a_lh.w, bw.z, bw.w);
-      }
-      if (lo_ok) {
-        const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&ylo);
-        *py_lo = lr_pack(__low2float(old) + c[0], __high2float(old) + c[1]);
-      }
-      if (hi_ok) {
-        const __nv_bfloat162 old = *reinterpret_cast<const __nv_bfloat162*>(&yhi);
-        *py_hi = lr_pack(__low2float(old) + c[2], __high2float(old) + c[3]);
-      }
-    }
-    __syncthreads();
-    // the new outputs leave as whole 16-byte vectors, a warp per row
-    const int yv = t_hi - t_lo;
-    for (int row = warp; row < nseq; row += LM_WARPS) {
-      if (active != nullptr && active[b0 + row] == 0) continue;
-      for (int v = lane; v < yv; v += 32)
-        *reinterpret_cast<uint4*>(yl + (size_t)row * d_out + (size_t)(t_lo + v) * 8) =
-            *reinterpret_cast<const uint4*>(ystage + (size_t)row * ys + v * 16);
+// grid = ceil(nl * B / 8) CTAs of 8 warps, a warp per (layer, sequence).  w_hi, w_lo [nl][B][G] bf16.
+template <int LPR>                   // lanes that share a state row: r = 4 * LPR
+__global__ void __launch_bounds__(LS_THREADS)
+k_lora_w(PtencDev p, int l0, int nl, const float* __restrict__ u_part, int n_part, __nv_bfloat16* __restrict__ w_hi,
+         __nv_bfloat16* __restrict__ w_lo) {
+  ls_let_next_start();
+  constexpr int r = 4 * LPR;
+  constexpr int SB = 8;                                        // 16-byte vectors of the state requested together
+  __shared__ __align__(16) float u_s[LS_WARPS][r];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int item = blockIdx.x * LS_WARPS + warp;
+  const int B = p.B, G = p.G;
+  const bool live = item < nl * B;
+  const int li = live ? item / B : 0, b = live ? item - li * B : 0;
+  const float4* Sv = reinterpret_cast<const float4*>(p.S + ((size_t)(l0 + li) * B + b) * G * r);
+  const int n_vec = G * r / 4;                                 // a multiple of 32: G is a multiple of 32
+  float4 sv[SB];
+#pragma unroll
+  for (int i = 0; i < SB; ++i)                                 // the state does not depend on the kernel in front
+    sv[i] = (live && i * 32 + lane < n_vec) ? Sv[i * 32 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+  ls_wait_for_previous();
+  if (live) {
+    for (int j = lane; j < r; j += 32) {
+      float v[PTENC_LORA_MAX_PART];                            // every part requested before the first is used
+#pragma unroll
+      for (int q = 0; q < PTENC_LORA_MAX_PART; ++q)
+        v[q] = q < n_part ? u_part[(((size_t)q * nl + li) * B + b) * r + j] : 0.f;
+      float t = 0.f;
+#pragma unroll
+      for (int q = 0; q < PTENC_LORA_MAX_PART; ++q) t += v[q];   // the same order in every launch
+      u_s[warp][j] = t;
     }
   }
+  __syncwarp();
+  if (!live) return;
+  const float4 uu = *reinterpret_cast<const float4*>(&u_s[warp][(lane % LPR) * 4]);
+  for (int v0 = 0; v0 < n_vec; v0 += SB * 32) {
+    if (v0 > 0) {
+#pragma unroll
+      for (int i = 0; i < SB; ++i)
+        sv[i] = (v0 + i * 32 + lane < n_vec) ? Sv[v0 + i * 32 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < SB; ++i) {
+      float d = fmaf(sv[i].x, uu.x, fmaf(sv[i].y, uu.y, fmaf(sv[i].z, uu.z, sv[i].w * uu.w)));
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      const int vec = v0 + i * 32 + lane;
+      if (vec < n_vec && (lane % LPR) == 0) {
+        const int g = vec / LPR;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(d);
+        w_hi[((size_t)li * B + b) * G + g] = hi;
+        w_lo[((size_t)li * B + b) * G + g] = __float2bfloat16_rn(d - __bfloat162float(hi));
+      }
+    }
+  }
+}
+
+// grid = (SO, nl).  Shared memory: the CTA's rows of A, one plane of 64-byte rows per 32 state rows, the four
+// 16-byte pieces of a row permuted by (row / 8) % 4 so that a fragment load touches every bank once.
+template <int KP>                    // G = 32 * KP
+__global__ void __launch_bounds__(LS_THREADS, 2)
+k_lora_y(PtencDev p, const __nv_bfloat16* __restrict__ A, __nv_bfloat16* __restrict__ y,
+         const __nv_bfloat16* __restrict__ w_hi, const __nv_bfloat16* __restrict__ w_lo,
+         const uint8_t* __restrict__ active, int d_out, int SO, int KS) {
+  extern __shared__ __align__(128) uint8_t ls_smem[];
+  constexpr int G = 32 * KP;
+  const int B = p.B;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qrow = lane >> 2, qcol = lane & 3;
+  const int li = blockIdx.y, so = blockIdx.x;
+  const int n_groups = (d_out + 31) >> 5;                      // groups of 32 outputs
+  const int g_lo = so * n_groups / SO, ng = (so + 1) * n_groups / SO - g_lo;
+  const int plane = ((n_groups + SO - 1) / SO) * 32 * 64;      // bytes of a plane
+  const __nv_bfloat16* Al = A + (size_t)li * d_out * G;
+  __nv_bfloat16* yl = y + (size_t)li * B * d_out;
+
+  for (int idx = tid; idx < ng * 32 * 4 * KP; idx += LS_THREADS) {
+    const int o_rel = idx / (4 * KP), ch = idx - o_rel * 4 * KP;
+    const int o = g_lo * 32 + o_rel;
+    uint8_t* dst = ls_smem + (size_t)(ch >> 2) * plane + o_rel * 64 + (((ch & 3) ^ ((o_rel >> 3) & 3)) << 4);
+    if (o < d_out) ls_cp16(dst, Al + (size_t)o * G + ch * 8);
+    else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+  }
+  ls_cp_commit();
+
+  const int n_mt = (B + 15) >> 4;
+  const int n_items = n_mt * KS;                               // (16 sequences, part of the CTA's groups) per warp pass
+  uint4 ya[LS_CB], yb[LS_CB];
+  auto request = [&](int item, int c0) {                       // the old outputs of up to LS_CB groups of an item
+    const int mt = item % n_mt, ks = item / n_mt;
+    const int c_hi = (ks + 1) * ng / KS;
+    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int i = 0; i < LS_CB; ++i) {
+      const int o = (g_lo + c0 + i) * 32 + qcol * 8;
+      const bool in = c0 + i < c_hi && o < d_out;
+      ya[i] = (in && b_lo < B) ? *reinterpret_cast<const uint4*>(yl + (size_t)b_lo * d_out + o) : zero;
+      yb[i] = (in && b_hi < B) ? *reinterpret_cast<const uint4*>(yl + (size_t)b_hi * d_out + o) : zero;
+    }
+  };
+  bool requested = false;
+  if (warp < n_items) { request(warp, (warp / n_mt) * ng / KS); requested = true; }   // in flight during the waits
+  ls_wait_for_previous();                                      // w is complete
+  ls_cp_wait_all();
+  __syncthreads();
+
+  for (int item = warp; item < n_items; item += LS_WARPS) {
+    const int mt = item % n_mt, ks = item / n_mt;
+    const int c_lo = ks * ng / KS, c_hi = (ks + 1) * ng / KS;
+    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
+    const bool st_lo = b_lo < B && (active == nullptr || active[b_lo] != 0);
+    const bool st_hi = b_hi < B && (active == nullptr || active[b_hi] != 0);
+    // the w fragments of the item's sixteen sequences
+    uint4 wh_l[KP], wh_h[KP], wl_l[KP], wl_h[KP];
+#pragma unroll
+    for (int k = 0; k < KP; ++k) {
+      const size_t o_lo = ((size_t)li * B + b_lo) * G + k * 32 + qcol * 8, o_hi = o_lo + (size_t)8 * G;
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+      wh_l[k] = b_lo < B ? *reinterpret_cast<const uint4*>(w_hi + o_lo) : zero;
+      wl_l[k] = b_lo < B ? *reinterpret_cast<const uint4*>(w_lo + o_lo) : zero;
+      wh_h[k] = b_hi < B ? *reinterpret_cast<const uint4*>(w_hi + o_hi) : zero;
+      wl_h[k] = b_hi < B ? *reinterpret_cast<const uint4*>(w_lo + o_hi) : zero;
+    }
+    // one group of 32 outputs for the item's sixteen sequences
+    auto group = [&](int cg, const uint4& old_lo, const uint4& old_hi) {
+      const int o = (g_lo + cg) * 32 + qcol * 8;
+      float c[4][4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0.f;
+        // column n of tile t is output 8 * (n / 2) + 2 * t + (n % 2) of the group: this lane's columns of the four
+        // tiles are eight consecutive outputs
+        const int o_rel = cg * 32 + 8 * (qrow >> 1) + 2 * t + (qrow & 1);
+#pragma unroll
+        for (int k = 0; k < KP; ++k) {
+          const uint4 aw = *reinterpret_cast<const uint4*>(ls_smem + (size_t)k * plane + o_rel * 64 +
+                                                           ((qcol ^ ((o_rel >> 3) & 3)) << 4));
+          lr_mma(c[t], wh_l[k].x, wh_h[k].x, wh_l[k].y, wh_h[k].y, aw.x, aw.y);
+          lr_mma(c[t], wh_l[k].z, wh_h[k].z, wh_l[k].w, wh_h[k].w, aw.z, aw.w);
+          lr_mma(c[t], wl_l[k].x, wl_h[k].x, wl_l[k].y, wl_h[k].y, aw.x, aw.y);
+          lr_mma(c[t], wl_l[k].z, wl_h[k].z, wl_l[k].w, wl_h[k].w, aw.z, aw.w);
+        }
+      }
+      if (o < d_out) {
+        const uint32_t ol[4] = {old_lo.x, old_lo.y, old_lo.z, old_lo.w}, oh[4] = {old_hi.x, old_hi.y, old_hi.z, old_hi.w};
+        uint32_t nlo[4], nhi[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&ol[t]);
+          const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&oh[t]);
+          nlo[t] = lr_pack(__low2float(a) + c[t][0], __high2float(a) + c[t][1]);
+          nhi[t] = lr_pack(__low2float(b2) + c[t][2], __high2float(b2) + c[t][3]);
+        }
+        if (st_lo) *reinterpret_cast<uint4*>(yl + (size_t)b_lo * d_out + o) = make_uint4(nlo[0], nlo[1], nlo[2], nlo[3]);
+        if (st_hi) *reinterpret_cast<uint4*>(yl + (size_t)b_hi * d_out + o) = make_uint4(nhi[0], nhi[1], nhi[2], nhi[3]);
+      }
+    };
+    for (int c0 = c_lo; c0 < c_hi; c0 += LS_CB) {
+      if (!requested) request(item, c0);
+      requested = false;
+#pragma unroll
+      for (int i = 0; i < LS_CB; ++i)
+        if (c0 + i < c_hi) group(c0 + i, ya[i], yb[i]);         // uniform over the warp
+    }
+  }
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t ls_launch(void (*kernel)(KArgs...), dim3 grid, size_t smem, bool after_previous, cudaStream_t st,
+                      Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(LS_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (after_previous) {
+    // programmatic dependent launch: the grid may become resident while the kernel in front of it on the stream
+    // (which signals that it allows this) is still running; the kernel waits before it reads that kernel's results
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+constexpr size_t LS_SMEM_MAX = 96 * 1024;   // per CTA, so that two CTAs fit an SM
+
+// The streaming path: bf16, r in {16, 32, 64}, G in {32, 64, 96, 128}, d_in a multiple of 32, d_out a multiple of 8.
+cudaError_t ls_apply(ptenc_cache* c, int l0, int nl, const __nv_bfloat16* A, const __nv_bfloat16* Bm,
+                     const __nv_bfloat16* x, __nv_bfloat16* y, const uint8_t* active, int d_in, int d_out,
+                     cudaStream_t st, bool* taken) {
+  const PtencDev& p = c->dev;
+  *taken = false;
+  if (c->cfg.dtype != PTENC_DTYPE_BF16 || (p.r != 16 && p.r != 32 && p.r != 64) || (p.G & 31) != 0 || p.G > 128 ||
+      (d_in & 31) != 0 || (d_out & 7) != 0 || nl > 65535)
+    return cudaSuccess;
+  static bool attr_done[PTENC_MAX_DEVICES] = {};
+  if (ptenc_first_use(attr_done, c->cfg.device)) {
+    cudaError_t e = cudaSuccess;
+    auto big = [&](const void* f) {
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LS_SMEM_MAX);
+    };
+    big((const void*)k_lora_u<2>); big((const void*)k_lora_u<4>); big((const void*)k_lora_u<8>);
+    big((const void*)k_lora_y<1>); big((const void*)k_lora_y<2>); big((const void*)k_lora_y<3>); big((const void*)k_lora_y<4>);
+    if (e != cudaSuccess) return e;
+  }
+  const int n_mt = (p.B + 15) / 16;
+  const int want = PTENC_LORA_CTAS_PER_SM * c->sm_count;        // CTAs of a streaming kernel: all resident at once
+  // slices of d_in: enough CTAs, a slice of B that fits shared memory, no more partial sums than the scratch holds
+  const int n_pairs = d_in >> 5;
+  int SL = want / nl;                                           // never a second, nearly empty wave
+  if (SL < 1) SL = 1;
+  if (SL > n_pairs) SL = n_pairs;
+  if (SL > PTENC_LORA_MAX_PART) SL = PTENC_LORA_MAX_PART;
+  while (SL < n_pairs && (size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL) > LS_SMEM_MAX) ++SL;
+  if (SL > PTENC_LORA_MAX_PART) return cudaSuccess;
+  int KS = LS_WARPS / n_mt;                                     // idle warps take parts of the slice
+  if (KS < 1) KS = 1;
+  if (SL * KS > PTENC_LORA_MAX_PART) KS = PTENC_LORA_MAX_PART / SL;
+  const size_t smem_u = (size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL);
+  // slices of d_out
+  const int n_groups = (d_out + 31) >> 5;
+  const int KP = p.G >> 5;
+  int SO = want / nl;
+  if (SO < 1) SO = 1;
+  if (SO > n_groups) SO = n_groups;
+  while (SO < n_groups && (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64 > LS_SMEM_MAX) ++SO;
+  const size_t smem_y = (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64;
+  if (smem_y > LS_SMEM_MAX) return cudaSuccess;
+  int KS2 = LS_WARPS / n_mt;
+  if (KS2 < 1) KS2 = 1;
+  *taken = true;
+  __nv_bfloat16* w_hi = c->lora_w;
+  __nv_bfloat16* w_lo = c->lora_w + (size_t)p.L * p.B * p.G;
+  const float* u_c = c->lora_u;
+  cudaError_t e;
+  switch (p.r) {
+    case 16: e = ls_launch(k_lora_u<2>, dim3(SL, nl), smem_u, false, st, p, Bm, x, c->lora_u, d_in, SL, KS); break;
+    case 32: e = ls_launch(k_lora_u<4>, dim3(SL, nl), smem_u, false, st, p, Bm, x, c->lora_u, d_in, SL, KS); break;
+    default: e = ls_launch(k_lora_u<8>, dim3(SL, nl), smem_u, false, st, p, Bm, x, c->lora_u, d_in, SL, KS); break;
+  }
+  c->launches++;
+  if (e != cudaSuccess) return e;
+  const dim3 gw((nl * p.B + LS_WARPS - 1) / LS_WARPS);
+  switch (p.r) {
+    case 16: e = ls_launch(k_lora_w<4>, gw, 0, true, st, p, l0, nl, u_c, SL * KS, w_hi, w_lo); break;
+    case 32: e = ls_launch(k_lora_w<8>, gw, 0, true, st, p, l0, nl, u_c, SL * KS, w_hi, w_lo); break;
+    default: e = ls_launch(k_lora_w<16>, gw, 0, true, st, p, l0, nl, u_c, SL * KS, w_hi, w_lo); break;
+  }
+  c->launches++;
+  if (e != cudaSuccess) return e;
+  const __nv_bfloat16* w_hi_c = w_hi;
+  const __nv_bfloat16* w_lo_c = w_lo;
+  switch (KP) {
+    case 1: e = ls_launch(k_lora_y<1>, dim3(SO, nl), smem_y, true, st, p, A, y, w_hi_c, w_lo_c, active, d_out, SO, KS2); break;
+    case 2: e = ls_launch(k_lora_y<2>, dim3(SO, nl), smem_y, true, st, p, A, y, w_hi_c, w_lo_c, active, d_out, SO, KS2); break;
+    case 3: e = ls_launch(k_lora_y<3>, dim3(SO, nl), smem_y, true, st, p, A, y, w_hi_c, w_lo_c, active, d_out, SO, KS2); break;
+    default: e = ls_launch(k_lora_y<4>, dim3(SO, nl), smem_y, true, st, p, A, y, w_hi_c, w_lo_c, active, d_out, SO, KS2); break;
+  }
+  c->launches++;
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
@@ -432,23 +541,11 @@ k_lora_apply_cluster(PtencDev p, int l0, const __nv_bfloat16* __restrict__ A, co
 cudaError_t ptenc_launch_lora_apply(ptenc_cache* c, int l0, int nl, const void* A, const void* Bm, const void* x,
                                     void* y, const uint8_t* active, int d_in, int d_out, cudaStream_t st) {
   const PtencDev& p = c->dev;
-  // tensor-core path: bf16, r a multiple of 8, G and d_in multiples of 32 (d_in at least 128: a slice per CTA of the
-  // cluster), d_out a multiple of 8, and slices that fit the staging buffer with two CTAs per SM
-  if (c->cfg.dtype == PTENC_DTYPE_BF16 && (p.r & 7) == 0 && (p.G & 31) == 0 && (d_in & 31) == 0 && d_in >= 128 &&
-      (d_out & 7) == 0 && lr_mma_smem(p.G, p.r, d_in, d_out) <= 100 * 1024 &&
-      (long long)nl * ((p.B + LM_SEQ - 1) / LM_SEQ) <= 65535) {
-    const size_t smem = lr_mma_smem(p.G, p.r, d_in, d_out);
-    static bool attr_done_c[PTENC_MAX_DEVICES] = {};
-    if (ptenc_first_use(attr_done_c, c->cfg.device)) {
-      cudaError_t e = cudaFuncSetAttribute(k_lora_apply_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-      if (e != cudaSuccess) return e;
-    }
-    const int nb = (p.B + LM_SEQ - 1) / LM_SEQ;
-    k_lora_apply_cluster<<<dim3(LM_CLUSTER, nl * nb), LM_THREADS, smem, st>>>(
-        p, l0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, active,
-        d_in, d_out);
-    c->launches++;
-    return cudaGetLastError();
+  {
+    bool taken = false;
+    cudaError_t e = ls_apply(c, l0, nl, (const __nv_bfloat16*)A, (const __nv_bfloat16*)Bm, (const __nv_bfloat16*)x,
+                             (__nv_bfloat16*)y, active, d_in, d_out, st, &taken);
+    if (taken || e != cudaSuccess) return e;
   }
   const size_t smem = sizeof(float) * ((((size_t)LR_SEQ * (p.r + p.G) + 3) & ~(size_t)3) +
                                        (((size_t)LR_SEQ * p.G * (p.r + 1) + 3) & ~(size_t)3)) +

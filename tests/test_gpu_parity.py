@@ -394,13 +394,15 @@ def test_prefill_misuse_sets_the_status_word():
     p.close()
 
 
-@pytest.mark.parametrize("dtype,G,r,d_in,d_out", [("bf16", 16, 24, 328, 200), ("fp32", 16, 24, 328, 200),
-                                                  ("bf16", 32, 32, 352, 200), ("bf16", 64, 16, 1024, 520)])
-def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out):
+@pytest.mark.parametrize("dtype,G,r,d_in,d_out,B", [("bf16", 16, 24, 328, 200, 11), ("fp32", 16, 24, 328, 200, 11),
+                                                    ("bf16", 32, 32, 352, 200, 11), ("bf16", 64, 16, 1024, 520, 11),
+                                                    ("bf16", 32, 32, 1792, 904, 37), ("bf16", 64, 64, 512, 264, 20),
+                                                    ("bf16", 128, 16, 256, 72, 16), ("bf16", 96, 32, 3584, 64, 130)])
+def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out, B):
     """y += A (S (B x)) with the state the rollout has produced so far, per sequence, against the oracle's
     (W + A S B) x written out; masked rows untouched; all layers in one call and one layer alone."""
     from oracle.ptenc_oracle import lora_apply
-    L, B = 2, 11      # the last two shape sets take the tensor-core kernel, the first two the shape-generic one
+    L = 2             # the first two shape sets take the shape-generic kernel, the others the tensor-core kernels
     p = Pair(pt, n_layers=L, batch=B, n_q_heads=4, n_kv_heads=2, head_dim=64, window=12, evict_chunk=3, dtype=dtype,
              seed=77, n_global=G, rank=r)
     for t in range(30):
@@ -409,7 +411,7 @@ def test_dynamic_weight_update_from_the_running_state(dtype, G, r, d_in, d_out):
     Bm = p.gen.generic(61, 0, (L, r, d_in), d_in ** -0.5)
     x = p.gen.generic(62, 0, (L, B, d_in), 1.0)
     y0 = p.gen.generic(63, 0, (L, B, d_out), 1.0)
-    active = torch.tensor([1, 1, 0, 1, 1, 1, 1, 0, 1, 1, 1], dtype=torch.uint8, device="cuda")
+    active = torch.tensor([0 if b % 7 == 2 else 1 for b in range(B)], dtype=torch.uint8, device="cuda")
     y = y0.clone()
     p.cache.lora_apply(-1, A, Bm, x, y, active)
     y1 = y0[1].clone()
