@@ -206,7 +206,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   // [4..8] ring state and tile enumeration of the unit (head, count, pinned, t0, len2); [9] first tile of the piece
   // in the unit's enumeration, [10] tiles of the piece; [11] pieces of the unit, [12] this piece, [13] first partial
   // slot of the unit (split units only)
-  __shared__ long long s_part[NTHREADS];
+  __shared__ long long s_part[NTHREADS / 32];
   __shared__ int s_items[NTHREADS + 1];
   __shared__ int s_split[NTHREADS + 1];
 
@@ -222,6 +222,10 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     misc[0] = 0; misc[1] = 0; misc[8] = 0; misc[9] = 0;
     desc[0] = 0; desc[16] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid == NW * 32) {                                      // the two tensor maps are wanted at the first tile
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmK)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmV)) : "memory");
   }
   for (int i = tid; i < 2 * SM::Q_BYTES / 4; i += NTHREADS) reinterpret_cast<uint32_t*>(smem + SM::OFF_Q)[i] = 0u;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -278,22 +282,45 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     return en;
   };
   auto load_entry = [&](int e) -> Entry { return make_entry(fetch(e), e); };
-  // every thread takes a contiguous chunk of the entries; tiles, items and pieces of split units per chunk
+  // every thread takes a contiguous chunk of the entries; tiles, items and pieces of split units per chunk.  This
+  // code runs once per launch, straight from instruction memory that the K/V stream of the launch before has pushed
+  // out of every cache: it is kept short (rolled loops, sums and prefixes through warp shuffles), and the second
+  // pass over the entries is skipped when no unit is split, which the first pass can tell.
   const int chunk = (n_ent + NTHREADS - 1) / NTHREADS;
   const int e_lo = min(tid * chunk, n_ent), e_hi = min(e_lo + chunk, n_ent);
+  constexpr int NWARPS = NTHREADS / 32;
+  // In the common launch -- every entry has tiles and no unit is split -- item i is simply (entry i / H_kv, head
+  // i % H_kv), and CTA c starts on item c: the ring words of that entry are requested now, with the first pass.
+  const Raw first_raw = fetch((int)blockIdx.x / Hkv);
   long long mine = 0;
+  int nz = 0, mx = 0;                                        // entries with tiles, longest entry
+#pragma unroll 1
   for (int e = e_lo; e < e_hi; e += 4) {                      // four entries' ring words requested at once
     Raw r[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) r[u] = fetch(e + u < e_hi ? e + u : e_hi - 1);
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (e + u < e_hi) mine += make_entry(r[u], e + u).nt;
+    for (int u = 0; u < 4; ++u) {
+      if (e + u < e_hi) {
+        const int nt = make_entry(r[u], e + u).nt;
+        mine += nt;
+        nz += nt > 0 ? 1 : 0;
+        mx = max(mx, nt);
+      }
+    }
   }
-  s_part[tid] = mine;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  __shared__ int s_wsum[3][NWARPS];
+  if (lane == 0) { s_part[warp] = mine; s_wsum[2][warp] = mx; }
   __syncthreads();
   long long total = 0;
-  for (int i = 0; i < NTHREADS; ++i) total += s_part[i];
+  int longest = 0;
+#pragma unroll
+  for (int i = 0; i < NWARPS; ++i) { total += s_part[i]; longest = max(longest, s_wsum[2][i]); }
   const long long T = total * Hkv;                     // tiles of the whole call
   // piece size: about `bal` items per CTA when the call is small; a unit is never cut finer than 8 tiles.  With
   // bal <= part_slots / (2 gridDim) the pieces of split units always fit the partial slots: a unit is split only if
@@ -304,30 +331,38 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   const int piece = (int)(piece_ll < 8 ? 8 : (piece_ll > (1 << 24) ? (1 << 24) : piece_ll));
   auto pieces_of = [&](int nt) -> int { return nt <= 0 ? 0 : (nt + piece - 1) / piece; };
   {
-    int items = 0, split = 0;
-    for (int e = e_lo; e < e_hi; ++e) {                       // the ring words are in L1 now
-      const int pc = pieces_of(load_entry(e).nt);
-      items += Hkv * pc;
-      if (pc > 1) split += Hkv * pc;
+    int items = Hkv * nz, split = 0;                          // no unit longer than a piece: every unit is one item
+    if (longest > piece) {                                    // uniform over the CTA
+      items = 0;
+#pragma unroll 1
+      for (int e = e_lo; e < e_hi; ++e) {                     // the ring words are in L1 or L2 now
+        const int pc = pieces_of(load_entry(e).nt);
+        items += Hkv * pc;
+        if (pc > 1) split += Hkv * pc;
+      }
     }
-    s_items[tid] = items;
-    s_split[tid] = split;
-  }
-  __syncthreads();
-  {
-    int bi = 0, bs = 0, ti = 0, ts = 0;
-    for (int i = 0; i < NTHREADS; ++i) {
-      const int vi = s_items[i], vs = s_split[i];
-      if (i < tid) { bi += vi; bs += vs; }
-      ti += vi; ts += vs;
+    // exclusive prefixes over the threads: inclusive scan inside the warp, then the warps' totals
+    int ci = items, cs = split;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, ci, o), c = __shfl_up_sync(0xffffffffu, cs, o);
+      if (lane >= o) { ci += a; cs += c; }
     }
+    if (lane == 31) { s_wsum[0][warp] = ci; s_wsum[1][warp] = cs; }
     __syncthreads();
+    int bi = ci - items, bs = cs - split, ti = 0, ts = 0;
+#pragma unroll
+    for (int w = 0; w < NWARPS; ++w) {
+      if (w < warp) { bi += s_wsum[0][w]; bs += s_wsum[1][w]; }
+      ti += s_wsum[0][w]; ts += s_wsum[1][w];
+    }
     s_items[tid] = bi;                                        // exclusive prefixes; the totals go last
     s_split[tid] = bs;
     if (tid == 0) { s_items[NTHREADS] = ti; s_split[NTHREADS] = ts; }
   }
   __syncthreads();
   const int n_items = s_items[NTHREADS];
+  const bool plain = longest <= piece && n_items == Hkv * n_ent;   // see above; uniform over the launch
 
   if (warp > NW) {
     // ================================================================ encoder warps (see the file header)
@@ -378,6 +413,12 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       pd.item = item; pd.tch = -1; pd.ce_lo = pd.ce_hi = 0;
       pd.raw.head = pd.raw.count = pd.raw.sink = pd.raw.act = 0; pd.raw.n = 0;
       if (item >= n_items) return pd;
+      if (plain) {                                           // no search: the entry follows from the item's number
+        pd.tch = -2;
+        pd.ce_lo = item / Hkv;
+        pd.raw = fetch(pd.ce_lo);
+        return pd;
+      }
       for (int base = 0; base < NTHREADS; base += 32) {
         const int idx = base + lane;
         const bool hit = idx < NTHREADS && s_items[idx] <= item && item < s_items[idx + 1];
@@ -396,6 +437,15 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       it.kind = 0; it.e = -1; it.h = it.k = it.iu_lo = it.n_mine = it.P = it.slot_base = 0;
       it.en.head = it.en.count = it.en.sink = it.en.nt = it.en.t0 = it.en.len2 = 0;
       if (pd.item >= n_items) { it.kind = 2; return it; }
+      if (pd.tch == -2) {
+        it.e = pd.ce_lo;
+        it.en = make_entry(pd.raw, it.e);
+        it.h = pd.item - it.e * Hkv;
+        it.P = 1;
+        it.n_mine = it.en.nt;
+        if (it.n_mine > 0) it.kind = 1;
+        return it;
+      }
       if (pd.tch < 0) return it;
       int rem = pd.item - s_items[pd.tch];
       int split_before = s_split[pd.tch];
@@ -440,12 +490,21 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       it.kind = 1;
       return it;
     };
-    auto grab = [&]() -> int { return lane == 0 ? atomicAdd(p.work, 1) : 0; };
+    // Item numbers: CTA c starts on item c without asking; the counter hands out gridDim.x, gridDim.x + 1, ...
+    auto grab = [&]() -> int { return lane == 0 ? atomicAdd(p.work, 1) + (int)gridDim.x : 0; };
+    const int last_grab = max(n_items, (int)gridDim.x) + (int)gridDim.x - 1;   // what the launch's last grab returns
 
-    int grabbed = grab();                                    // number of the first item
-    Item cur = lookup_finish(lookup_begin(__shfl_sync(0xffffffffu, grabbed, 0)));
-    if (cur.kind == 1) grabbed = grab();                     // every CTA makes exactly one grab that finds nothing left
+    Pending pd;
+    if (plain && (int)blockIdx.x < n_items) {                // the first item's ring words are here already
+      pd.item = (int)blockIdx.x; pd.tch = -2; pd.ce_lo = (int)blockIdx.x / Hkv; pd.ce_hi = 0;
+      pd.raw = first_raw;
+    } else {
+      pd = lookup_begin((int)blockIdx.x);
+    }
+    int grabbed = grab();                                    // the item after that; every CTA makes exactly one grab
+                                                             // that finds nothing left (this one, if it has no item)
     while (!aborted) {
+      const Item cur = lookup_finish(pd);
       const uint32_t ubuf = useq & 1;
       volatile int* dsc = desc + ubuf * 16;
       if (cur.kind != 1) {
@@ -456,7 +515,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         }
         // nothing left: tell the consumers, and the CTA whose grab was the very last of the launch rewinds the counter
         if (lane == 0) {
-          if (grabbed == n_items + (int)gridDim.x - 1) *p.work = 0;
+          if (grabbed == last_grab) *p.work = 0;
           if (mbar_wait(bar_qempty + 8 * ubuf, ((useq >> 1) & 1) ^ 1)) {
             dsc[0] = 2;
             mbar_arrive(bar_qfull + 8 * ubuf);
@@ -484,7 +543,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
       }
       // the next item: its number has arrived by now; request its entries' ring words, and the number after it
       const int item2 = __shfl_sync(0xffffffffu, grabbed, 0);
-      const Pending pd = lookup_begin(item2);
+      pd = lookup_begin(item2);
       if (item2 < n_items) grabbed = grab();
       aborted = __shfl_sync(0xffffffffu, aborted ? 1 : 0, 0) != 0;
       if (lane < NW && !aborted) {
@@ -512,7 +571,6 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
         }
       }
       aborted = __any_sync(0xffffffffu, aborted);
-      cur = lookup_finish(pd);
       ++useq;
     }
     aborted = __any_sync(0xffffffffu, aborted);
