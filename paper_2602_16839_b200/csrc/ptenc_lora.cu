@@ -165,13 +165,11 @@ k_lora_apply(PtencDev p, int l0, const T* __restrict__ A, const T* __restrict__ 
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int LS_THREADS = 256;
 constexpr int LS_WARPS = LS_THREADS / 32;
-#ifndef PTENC_LORA_CB
-#define PTENC_LORA_CB 6
-#endif
 #ifndef PTENC_LORA_CTAS_PER_SM
 #define PTENC_LORA_CTAS_PER_SM 2
 #endif
-constexpr int LS_CB = PTENC_LORA_CB; // 32-wide chunks of the contraction / 32-wide groups of outputs requested together
+constexpr int LS_SLOTS = 8;          // 32-wide chunks of the contraction / 32-wide groups of outputs a warp keeps in flight
+constexpr int LS_SLOT_BYTES = LS_WARPS * LS_SLOTS * 2 * 32 * 16;   // per CTA: [warp][slot][row half][lane] 16 bytes
 
 __device__ __forceinline__ void lr_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -190,6 +188,9 @@ __device__ __forceinline__ void ls_cp16(void* smem_dst, const void* gsrc) {
 }
 __device__ __forceinline__ void ls_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void ls_cp_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void ls_cp_wait_but() {      // all but the N most recent groups have landed
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
 __device__ __forceinline__ void ls_let_next_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void ls_wait_for_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -218,52 +219,75 @@ k_lora_u(PtencDev p, const __nv_bfloat16* __restrict__ Bm, const __nv_bfloat16* 
     for (int v = lane; v < np * 4; v += 32) ls_cp16(ls_smem + (size_t)row * rs + v * 16, Bl + (size_t)row * d_in + v * 8);
   ls_cp_commit();
 
+  // The streaming part is written as short rolled loops: a launch runs its code once, from instruction memory that
+  // is in no cache, so every unrolled copy costs more than the loop overhead it saves.  A lane's 16-byte pieces
+  // travel by asynchronous copy into shared-memory slots that only this lane reads (no barrier), LS_SLOTS chunks
+  // ahead of the mma; one copy group is committed per chunk, empty past the end, so that "all but the LS_SLOTS - 1
+  // most recent groups" always means "the chunk that is needed next".
   const int n_mt = (B + 15) >> 4;
   const int n_items = n_mt * KS;                               // (16 sequences, part of the slice) per warp pass
-  uint4 xa[LS_CB], xb[LS_CB];
-  auto request = [&](int item, int c0) {                       // the inputs of up to LS_CB chunks of an item
+  uint4* slots = reinterpret_cast<uint4*>(ls_smem + (((size_t)r * rs + 127) & ~(size_t)127)) + warp * (LS_SLOTS * 2 * 32) + lane;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  int item = warp;
+  int c_lo = 0, c_hi = 0, b_lo = 0;
+  const __nv_bfloat16* src_lo = xl;
+  const __nv_bfloat16* src_hi = xl;
+  auto open_item = [&]() {                                     // this warp's next item and its first LS_SLOTS chunks
     const int mt = item % n_mt, ks = item / n_mt;
-    const int c_hi = (ks + 1) * np / KS;
-    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
-    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-    for (int i = 0; i < LS_CB; ++i) {
-      const bool in = c0 + i < c_hi;
-      xa[i] = (in && b_lo < B) ? __ldg(reinterpret_cast<const uint4*>(xl + (size_t)b_lo * d_in + (c0 + i) * 32 + qcol * 8)) : zero;
-      xb[i] = (in && b_hi < B) ? __ldg(reinterpret_cast<const uint4*>(xl + (size_t)b_hi * d_in + (c0 + i) * 32 + qcol * 8)) : zero;
-    }
+    c_lo = ks * np / KS;
+    c_hi = (ks + 1) * np / KS;
+    b_lo = 16 * mt + qrow;
+    src_lo = xl + (size_t)b_lo * d_in + qcol * 8;
+    src_hi = src_lo + (size_t)8 * d_in;
   };
-  bool requested = false;
-  if (warp < n_items) { request(warp, (warp / n_mt) * np / KS); requested = true; }   // in flight while B lands
-  ls_cp_wait_all();
+  auto request = [&](int c, int slot) {                        // chunk c of the item into a slot; one group either way
+    if (c < c_hi) {
+      if (b_lo < B) ls_cp16(slots + (2 * slot) * 32, src_lo + c * 32); else slots[(2 * slot) * 32] = zero;
+      if (b_lo + 8 < B) ls_cp16(slots + (2 * slot + 1) * 32, src_hi + c * 32); else slots[(2 * slot + 1) * 32] = zero;
+    }
+    ls_cp_commit();
+  };
+  bool have = item < n_items;
+  if (have) {
+    open_item();
+#pragma unroll 1
+    for (int i = 0; i < LS_SLOTS; ++i) request(c_lo + i, i);
+    ls_cp_wait_but<LS_SLOTS>();                                // the slice of B (the oldest group) has landed
+  } else {
+    ls_cp_wait_all();
+  }
   __syncthreads();
 
-  for (int item = warp; item < n_items; item += LS_WARPS) {
-    const int mt = item % n_mt, ks = item / n_mt;
-    const int c_lo = ks * np / KS, c_hi = (ks + 1) * np / KS;
+  while (have) {
     float acc[NT][4];
 #pragma unroll
     for (int t = 0; t < NT; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
-    for (int c0 = c_lo; c0 < c_hi; c0 += LS_CB) {
-      if (!requested) request(item, c0);
-      requested = false;
+#pragma unroll 1
+    for (int c = c_lo; c < c_hi; ++c) {
+      const int slot = (c - c_lo) % LS_SLOTS;
+      ls_cp_wait_but<LS_SLOTS - 1>();
+      const uint4 xa = slots[(2 * slot) * 32], xb = slots[(2 * slot + 1) * 32];
 #pragma unroll
-      for (int i = 0; i < LS_CB; ++i) {
-        if (c0 + i < c_hi) {
-#pragma unroll
-          for (int t = 0; t < NT; ++t) {
-            const uint4 bw = *reinterpret_cast<const uint4*>(ls_smem + (size_t)(t * 8 + qrow) * rs + (c0 + i) * 64 + qcol * 16);
-            lr_mma(acc[t], xa[i].x, xb[i].x, xa[i].y, xb[i].y, bw.x, bw.y);
-            lr_mma(acc[t], xa[i].z, xb[i].z, xa[i].w, xb[i].w, bw.z, bw.w);
-          }
-        }
+      for (int t = 0; t < NT; ++t) {
+        const uint4 bw = *reinterpret_cast<const uint4*>(ls_smem + (size_t)(t * 8 + qrow) * rs + c * 64 + qcol * 16);
+        lr_mma(acc[t], xa.x, xb.x, xa.y, xb.y, bw.x, bw.y);
+        lr_mma(acc[t], xa.z, xb.z, xa.w, xb.w, bw.z, bw.w);
       }
+      request(c + LS_SLOTS, slot);
     }
+    const int mt = item % n_mt, ks = item / n_mt;
     float* dst = u_part + (((size_t)(sl * KS + ks) * nl + li) * B + 16 * mt + qrow) * r + 2 * qcol;
 #pragma unroll
     for (int t = 0; t < NT; ++t) {
-      if (16 * mt + qrow < B) *reinterpret_cast<float2*>(dst + t * 8) = make_float2(acc[t][0], acc[t][1]);
-      if (16 * mt + qrow + 8 < B) *reinterpret_cast<float2*>(dst + (size_t)8 * r + t * 8) = make_float2(acc[t][2], acc[t][3]);
+      if (b_lo < B) *reinterpret_cast<float2*>(dst + t * 8) = make_float2(acc[t][0], acc[t][1]);
+      if (b_lo + 8 < B) *reinterpret_cast<float2*>(dst + (size_t)8 * r + t * 8) = make_float2(acc[t][2], acc[t][3]);
+    }
+    item += LS_WARPS;
+    have = item < n_items;
+    if (have) {
+      open_item();
+#pragma unroll 1
+      for (int i = 0; i < LS_SLOTS; ++i) request(c_lo + i, i);
     }
   }
 }
@@ -354,63 +378,76 @@ k_lora_y(PtencDev p, const __nv_bfloat16* __restrict__ A, __nv_bfloat16* __restr
   }
   ls_cp_commit();
 
+  // rolled loops and lane-private slots as in k_lora_u: the old outputs of a group of 32 columns travel LS_SLOTS groups
+  // ahead of the mma, one copy group per group of outputs
   const int n_mt = (B + 15) >> 4;
   const int n_items = n_mt * KS;                               // (16 sequences, part of the CTA's groups) per warp pass
-  uint4 ya[LS_CB], yb[LS_CB];
-  auto request = [&](int item, int c0) {                       // the old outputs of up to LS_CB groups of an item
+  uint4* slots = reinterpret_cast<uint4*>(ls_smem + (size_t)KP * plane) + warp * (LS_SLOTS * 2 * 32) + lane;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  int item = warp;
+  int c_lo = 0, c_hi = 0, b_lo = 0;
+  __nv_bfloat16* row_lo = yl;
+  __nv_bfloat16* row_hi = yl;
+  auto open_item = [&]() {
     const int mt = item % n_mt, ks = item / n_mt;
-    const int c_hi = (ks + 1) * ng / KS;
-    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
-    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-    for (int i = 0; i < LS_CB; ++i) {
-      const int o = (g_lo + c0 + i) * 32 + qcol * 8;
-      const bool in = c0 + i < c_hi && o < d_out;
-      ya[i] = (in && b_lo < B) ? *reinterpret_cast<const uint4*>(yl + (size_t)b_lo * d_out + o) : zero;
-      yb[i] = (in && b_hi < B) ? *reinterpret_cast<const uint4*>(yl + (size_t)b_hi * d_out + o) : zero;
-    }
+    c_lo = ks * ng / KS;
+    c_hi = (ks + 1) * ng / KS;
+    b_lo = 16 * mt + qrow;
+    row_lo = yl + (size_t)b_lo * d_out + qcol * 8;
+    row_hi = row_lo + (size_t)8 * d_out;
   };
-  bool requested = false;
-  if (warp < n_items) { request(warp, (warp / n_mt) * ng / KS); requested = true; }   // in flight during the waits
+  auto request = [&](int c, int slot) {                        // group c of the item's old outputs; one copy group either way
+    const int o = (g_lo + c) * 32;
+    if (c < c_hi && o + qcol * 8 < d_out) {
+      if (b_lo < B) ls_cp16(slots + (2 * slot) * 32, row_lo + o); else slots[(2 * slot) * 32] = zero;
+      if (b_lo + 8 < B) ls_cp16(slots + (2 * slot + 1) * 32, row_hi + o); else slots[(2 * slot + 1) * 32] = zero;
+    }
+    ls_cp_commit();
+  };
+  bool have = item < n_items;
+  if (have) {
+    open_item();
+#pragma unroll 1
+    for (int i = 0; i < LS_SLOTS; ++i) request(c_lo + i, i);   // in flight during the waits
+  }
   ls_wait_for_previous();                                      // w is complete
-  ls_cp_wait_all();
+  if (have) ls_cp_wait_but<LS_SLOTS>(); else ls_cp_wait_all(); // the rows of A (the oldest group) have landed
   __syncthreads();
 
-  for (int item = warp; item < n_items; item += LS_WARPS) {
-    const int mt = item % n_mt, ks = item / n_mt;
-    const int c_lo = ks * ng / KS, c_hi = (ks + 1) * ng / KS;
-    const int b_lo = 16 * mt + qrow, b_hi = b_lo + 8;
+  while (have) {
     const bool st_lo = b_lo < B && (active == nullptr || active[b_lo] != 0);
-    const bool st_hi = b_hi < B && (active == nullptr || active[b_hi] != 0);
+    const bool st_hi = b_lo + 8 < B && (active == nullptr || active[b_lo + 8] != 0);
     // the w fragments of the item's sixteen sequences
     uint4 wh_l[KP], wh_h[KP], wl_l[KP], wl_h[KP];
 #pragma unroll
     for (int k = 0; k < KP; ++k) {
       const size_t o_lo = ((size_t)li * B + b_lo) * G + k * 32 + qcol * 8, o_hi = o_lo + (size_t)8 * G;
-      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
       wh_l[k] = b_lo < B ? *reinterpret_cast<const uint4*>(w_hi + o_lo) : zero;
       wl_l[k] = b_lo < B ? *reinterpret_cast<const uint4*>(w_lo + o_lo) : zero;
-      wh_h[k] = b_hi < B ? *reinterpret_cast<const uint4*>(w_hi + o_hi) : zero;
-      wl_h[k] = b_hi < B ? *reinterpret_cast<const uint4*>(w_lo + o_hi) : zero;
+      wh_h[k] = b_lo + 8 < B ? *reinterpret_cast<const uint4*>(w_hi + o_hi) : zero;
+      wl_h[k] = b_lo + 8 < B ? *reinterpret_cast<const uint4*>(w_lo + o_hi) : zero;
     }
-    // one group of 32 outputs for the item's sixteen sequences
-    auto group = [&](int cg, const uint4& old_lo, const uint4& old_hi) {
-      const int o = (g_lo + cg) * 32 + qcol * 8;
-      float c[4][4];
+#pragma unroll 1
+    for (int c = c_lo; c < c_hi; ++c) {
+      const int slot = (c - c_lo) % LS_SLOTS;
+      ls_cp_wait_but<LS_SLOTS - 1>();
+      const uint4 old_lo = slots[(2 * slot) * 32], old_hi = slots[(2 * slot + 1) * 32];
+      const int o = (g_lo + c) * 32 + qcol * 8;
+      float acc[4][4];
 #pragma unroll
       for (int t = 0; t < 4; ++t) {
-        c[t][0] = c[t][1] = c[t][2] = c[t][3] = 0.f;
+        acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
         // column n of tile t is output 8 * (n / 2) + 2 * t + (n % 2) of the group: this lane's columns of the four
         // tiles are eight consecutive outputs
-        const int o_rel = cg * 32 + 8 * (qrow >> 1) + 2 * t + (qrow & 1);
+        const int o_rel = c * 32 + 8 * (qrow >> 1) + 2 * t + (qrow & 1);
 #pragma unroll
         for (int k = 0; k < KP; ++k) {
           const uint4 aw = *reinterpret_cast<const uint4*>(ls_smem + (size_t)k * plane + o_rel * 64 +
                                                            ((qcol ^ ((o_rel >> 3) & 3)) << 4));
-          lr_mma(c[t], wh_l[k].x, wh_h[k].x, wh_l[k].y, wh_h[k].y, aw.x, aw.y);
-          lr_mma(c[t], wh_l[k].z, wh_h[k].z, wh_l[k].w, wh_h[k].w, aw.z, aw.w);
-          lr_mma(c[t], wl_l[k].x, wl_h[k].x, wl_l[k].y, wl_h[k].y, aw.x, aw.y);
-          lr_mma(c[t], wl_l[k].z, wl_h[k].z, wl_l[k].w, wl_h[k].w, aw.z, aw.w);
+          lr_mma(acc[t], wh_l[k].x, wh_h[k].x, wh_l[k].y, wh_h[k].y, aw.x, aw.y);
+          lr_mma(acc[t], wh_l[k].z, wh_h[k].z, wh_l[k].w, wh_h[k].w, aw.z, aw.w);
+          lr_mma(acc[t], wl_l[k].x, wl_h[k].x, wl_l[k].y, wl_h[k].y, aw.x, aw.y);
+          lr_mma(acc[t], wl_l[k].z, wl_h[k].z, wl_l[k].w, wl_h[k].w, aw.z, aw.w);
         }
       }
       if (o < d_out) {
@@ -418,21 +455,22 @@ k_lora_y(PtencDev p, const __nv_bfloat16* __restrict__ A, __nv_bfloat16* __restr
         uint32_t nlo[4], nhi[4];
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&ol[t]);
-          const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&oh[t]);
-          nlo[t] = lr_pack(__low2float(a) + c[t][0], __high2float(a) + c[t][1]);
-          nhi[t] = lr_pack(__low2float(b2) + c[t][2], __high2float(b2) + c[t][3]);
+          const __nv_bfloat162 va = *reinterpret_cast<const __nv_bfloat162*>(&ol[t]);
+          const __nv_bfloat162 vb = *reinterpret_cast<const __nv_bfloat162*>(&oh[t]);
+          nlo[t] = lr_pack(__low2float(va) + acc[t][0], __high2float(va) + acc[t][1]);
+          nhi[t] = lr_pack(__low2float(vb) + acc[t][2], __high2float(vb) + acc[t][3]);
         }
-        if (st_lo) *reinterpret_cast<uint4*>(yl + (size_t)b_lo * d_out + o) = make_uint4(nlo[0], nlo[1], nlo[2], nlo[3]);
-        if (st_hi) *reinterpret_cast<uint4*>(yl + (size_t)b_hi * d_out + o) = make_uint4(nhi[0], nhi[1], nhi[2], nhi[3]);
+        if (st_lo) *reinterpret_cast<uint4*>(row_lo + (g_lo + c) * 32) = make_uint4(nlo[0], nlo[1], nlo[2], nlo[3]);
+        if (st_hi) *reinterpret_cast<uint4*>(row_hi + (g_lo + c) * 32) = make_uint4(nhi[0], nhi[1], nhi[2], nhi[3]);
       }
-    };
-    for (int c0 = c_lo; c0 < c_hi; c0 += LS_CB) {
-      if (!requested) request(item, c0);
-      requested = false;
-#pragma unroll
-      for (int i = 0; i < LS_CB; ++i)
-        if (c0 + i < c_hi) group(c0 + i, ya[i], yb[i]);         // uniform over the warp
+      request(c + LS_SLOTS, slot);
+    }
+    item += LS_WARPS;
+    have = item < n_items;
+    if (have) {
+      open_item();
+#pragma unroll 1
+      for (int i = 0; i < LS_SLOTS; ++i) request(c_lo + i, i);
     }
   }
 }
@@ -458,7 +496,7 @@ cudaError_t ls_launch(void (*kernel)(KArgs...), dim3 grid, size_t smem, bool aft
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-constexpr size_t LS_SMEM_MAX = 96 * 1024;   // per CTA, so that two CTAs fit an SM
+constexpr size_t LS_SMEM_MAX = 112 * 1024;  // per CTA, so that two CTAs fit an SM
 
 // The streaming path: bf16, r in {16, 32, 64}, G in {32, 64, 96, 128}, d_in a multiple of 32, d_out a multiple of 8.
 cudaError_t ls_apply(ptenc_cache* c, int l0, int nl, const __nv_bfloat16* A, const __nv_bfloat16* Bm,
@@ -487,20 +525,21 @@ cudaError_t ls_apply(ptenc_cache* c, int l0, int nl, const __nv_bfloat16* A, con
   if (SL < 1) SL = 1;
   if (SL > n_pairs) SL = n_pairs;
   if (SL > PTENC_LORA_MAX_PART) SL = PTENC_LORA_MAX_PART;
-  while (SL < n_pairs && (size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL) > LS_SMEM_MAX) ++SL;
+  while (SL < n_pairs && (size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL) + 128 + LS_SLOT_BYTES > LS_SMEM_MAX) ++SL;
   if (SL > PTENC_LORA_MAX_PART) return cudaSuccess;
   int KS = LS_WARPS / n_mt;                                     // idle warps take parts of the slice
   if (KS < 1) KS = 1;
   if (SL * KS > PTENC_LORA_MAX_PART) KS = PTENC_LORA_MAX_PART / SL;
-  const size_t smem_u = (size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL);
+  const size_t smem_u = (((size_t)p.r * ls_b_stride((n_pairs + SL - 1) / SL) + 127) & ~(size_t)127) + LS_SLOT_BYTES;
+  if (smem_u > LS_SMEM_MAX) return cudaSuccess;
   // slices of d_out
   const int n_groups = (d_out + 31) >> 5;
   const int KP = p.G >> 5;
   int SO = want / nl;
   if (SO < 1) SO = 1;
   if (SO > n_groups) SO = n_groups;
-  while (SO < n_groups && (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64 > LS_SMEM_MAX) ++SO;
-  const size_t smem_y = (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64;
+  while (SO < n_groups && (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64 + LS_SLOT_BYTES > LS_SMEM_MAX) ++SO;
+  const size_t smem_y = (size_t)KP * ((n_groups + SO - 1) / SO) * 32 * 64 + LS_SLOT_BYTES;
   if (smem_y > LS_SMEM_MAX) return cudaSuccess;
   int KS2 = LS_WARPS / n_mt;
   if (KS2 < 1) KS2 = 1;
