@@ -19,18 +19,27 @@ constexpr int RE_WARPS = 8;                // (layer, sequence) pairs per CTA
 __global__ void __launch_bounds__(RE_WARPS * 32)
 k_ring_e1(PtencDev p, int l0, int nl, const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
           const uint8_t* __restrict__ active) {
-  // the attention launch behind this kernel may become resident and run its set-up now; it waits for this whole
-  // grid before it reads anything
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * RE_WARPS + (threadIdx.x >> 5);
-  if (item >= nl * p.B) return;
-  const int li = item / p.B, b = item - li * p.B;
+  const bool live = item < nl * p.B;
+  const int li = live ? item / p.B : 0, b = live ? item - li * p.B : 0;
   const size_t lb = (size_t)(l0 + li) * p.B + b;
   const size_t ob = (size_t)li * p.B + b;
   const int W = p.W, Hkv = p.Hkv;
   const int vph = p.D >> 3;                          // 16-byte vectors per (token, head) row
   const int vpr = p.d_kv >> 3;                       // and per token (all KV heads)
+  // the attention launch behind this kernel may become resident and run its set-up now; it waits for this whole
+  // grid before it reads anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!live) return;
+  // the arriving row does not depend on the ring state: its first two vectors per lane are requested with the ring words
+  uint4 nk0 = make_uint4(0u, 0u, 0u, 0u), nv0 = nk0, nk1 = nk0, nv1 = nk0;
+  {
+    const char* kn = reinterpret_cast<const char*>(k_new) + ob * (size_t)p.d_kv * 2;
+    const char* vn = reinterpret_cast<const char*>(v_new) + ob * (size_t)p.d_kv * 2;
+    if (lane < vpr) { nk0 = *reinterpret_cast<const uint4*>(kn + (size_t)lane * 16); nv0 = *reinterpret_cast<const uint4*>(vn + (size_t)lane * 16); }
+    if (lane + 32 < vpr) { nk1 = *reinterpret_cast<const uint4*>(kn + (size_t)(lane + 32) * 16); nv1 = *reinterpret_cast<const uint4*>(vn + (size_t)(lane + 32) * 16); }
+  }
 
   // every lane reads the ring state itself (same addresses: one request), so nothing waits for a broadcast
   const int act = (active == nullptr) ? 1 : (int)active[b];
@@ -60,9 +69,11 @@ k_ring_e1(PtencDev p, int l0, int nl, const __nv_bfloat16* __restrict__ k_new, c
   new_slot += ns;
   for (int v = lane; v < vpr; v += 32) {
     const int h = v / vph, vv = v - h * vph;
-    const size_t src_new = ((ob * Hkv + h) * p.D) * 2 + (size_t)vv * 16;
-    const uint4 nk = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(k_new) + src_new);
-    const uint4 nv = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(v_new) + src_new);
+    const size_t src_new = ((ob * Hkv + h) * p.D) * 2 + (size_t)vv * 16;      // = (ob * d_kv) * 2 + v * 16
+    const uint4 nk = v == lane ? nk0 : v == lane + 32 ? nk1
+                               : *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(k_new) + src_new);
+    const uint4 nv = v == lane ? nv0 : v == lane + 32 ? nv1
+                               : *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(v_new) + src_new);
     if (m) {
       // the evicted row is read by the lane that overwrites the same bytes below, so the read comes first
       const size_t src = (((lb * Hkv + h) * W + ev_slot) * p.D) * 2 + (size_t)vv * 16;
