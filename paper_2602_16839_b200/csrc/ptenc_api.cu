@@ -130,18 +130,21 @@ cudaError_t launch_append(ptenc_cache* c, int l0, int nl, const void* k_new, con
   return ptenc_launch_append_evict(c, l0, nl, k_new, v_new, active, slot_out, evict_first_out, n_evicted_out, st);
 }
 
-// True when a decode step on this cache runs as "append/evict alone, then the attention kernel with its spare warp
-// folding the staged rows": ring-per-step mode under the sliding-window policy on the tensor-core kernels.
+// True when a decode step on this cache runs as "append/evict alone, then the attention kernel with its spare warps
+// folding the staged rows": ring-per-step mode on the tensor-core kernels, under either eviction policy (both leave
+// the evicted row of a sequence in the same staging slot).
 bool step_folds_in_attention(const ptenc_cache* c) {
-  return c->cfg.policy == PTENC_POLICY_FIFO && c->cfg.encode_enabled && c->fast_attn &&
-         ptenc_step_e1_usable(c, nullptr, 0);
+  return c->cfg.encode_enabled && c->fast_attn && ptenc_step_e1_usable(c, nullptr, 0);
 }
 
 // a1 (+ a3 unless the attention launch of the step does it, see above) of a decode step.
 bool launch_append_and_encode(ptenc_cache* c, int l0, int nl, const void* k_new, const void* v_new,
                               const uint8_t* active, cudaStream_t st) {
-  if (step_folds_in_attention(c))
+  if (step_folds_in_attention(c)) {
+    if (c->cfg.policy == PTENC_POLICY_SCORE)
+      return ok(launch_append(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st), "decode_step/append_evict", st);
     return ok(ptenc_launch_ring_e1(c, l0, nl, k_new, v_new, active, st), "decode_step/append_evict", st);
+  }
   if (!ok(launch_append(c, l0, nl, k_new, v_new, active, nullptr, nullptr, nullptr, st), "decode_step/append_evict", st))
     return false;
   if (c->cfg.encode_enabled)
