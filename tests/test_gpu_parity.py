@@ -573,3 +573,30 @@ def test_launch_info_reports_the_instantiation():
     gen = pt.Cache(pt.make_config(n_layers=1, batch=2, n_q_heads=4, n_kv_heads=1, head_dim=64, window=64, dtype="fp32"))
     assert gen.attn_launch_info(-1) == {"consumer_warps": 0, "tile_tokens": 0, "stages": 0}
     gen.close()
+
+
+def test_a_step_with_every_sequence_inactive_changes_nothing_and_leaves_the_counters_clean():
+    """A launch with no work at all (every sequence masked out): outputs untouched, rings and states unchanged, status
+    clean -- and the launches after it behave as if it had not happened (the attention kernel's work counter and its
+    split-unit tickets are back at zero), on both instantiations."""
+    for warps in (0, 3):
+        p = Pair(pt, n_layers=2, batch=5, n_q_heads=8, n_kv_heads=2, head_dim=128, window=40, dtype="bf16", seed=9,
+                 attn_consumer_warps=warps)
+        for t in range(44):
+            p.step(t)
+        S_before = [p.cache.get_state(l).clone() for l in range(2)]
+        ring_before = [tuple(x.clone() for x in p.cache.get_ring(l)) for l in range(2)]
+        q = p.gen.step_q(44)
+        k, v = p.gen.step_kv(44)
+        out = torch.full_like(q, 7.0)
+        none = torch.zeros(5, dtype=torch.uint8, device="cuda")
+        p.cache.decode_step(-1, q, k, v, out, none)
+        assert torch.equal(out, torch.full_like(q, 7.0))
+        for l in range(2):
+            assert torch.equal(p.cache.get_state(l), S_before[l])
+            assert all(torch.equal(a, b) for a, b in zip(p.cache.get_ring(l), ring_before[l]))
+        assert p.cache.status() == 0
+        for t in range(44, 50):                            # ordinary steps afterwards, checked against the oracle
+            p.step(t)
+        assert p.cache.status() == 0
+        p.close()
