@@ -72,7 +72,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes moved (read + written, ncu counters) per algorithmic byte of the tensor-core attention kernel, keyed by
 # window: each ratio was measured on a launch with a smaller batch of the same head shape and window, and DRAM
 # traffic grows in proportion to the K/V tiles a launch reads.  Windows with no capture report no traffic figure.
-ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {512: 1.0132, 2048: 1.0057}
+ATTN_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {512: 1.0134, 2048: 1.0056}
 
 
 def workload_cfg(name: str) -> dict:
