@@ -5,7 +5,7 @@
 // registers, the 2r dot products against the encoder weights stream the weights from L2 with 16-byte loads, and the
 // rank-1 update of the [G, r] state runs a state row per lane.  Everything is fp32 except the stored rows and weights.
 //
-// The routine is the same wherever ring-per-step encoding happens -- in the spare warp of the attention kernel, where
+// The routine is the same wherever ring-per-step encoding happens -- on the spare warps of the attention kernel, where
 // it overlaps the K/V stream of the same step, and in the stand-alone kernel behind ptenc_encode -- so the fused step
 // and the separate calls give bit-identical states.
 #pragma once

@@ -108,7 +108,7 @@ cudaError_t ptenc_launch_set_encoder(ptenc_cache* c, int layer, const void* Wq, 
                                      const void* kg, const void* vg, cudaStream_t st);
 cudaError_t ptenc_launch_attn_generic(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active,
                                       void* out, float* lse, cudaStream_t st);
-// fold_staged: the kernel's spare warp also folds the rows staged by the append of the same step (E = 1) into the
+// fold_staged: the kernel's spare warps also fold the rows staged by the append of the same step (E = 1) into the
 // states of the layers of the call, while the K/V stream runs.
 // early: the launch directly follows ptenc_launch_ring_e1 on the same stream and may start while that kernel runs
 // (programmatic dependent launch); the attention kernel waits for it before its first read.

@@ -5,7 +5,7 @@
 //                  when the ring is full -- its row goes to the staging area -- writes the arriving token into the
 //                  freed slot and advances the ring.  This is all the attention of the same step depends on; it is a
 //                  chain of two memory round trips, so the fused decode step runs it alone in front of the attention
-//                  kernel and lets the attention kernel's spare warp fold the staged rows (a3) while the K/V stream
+//                  kernel and lets the attention kernel's spare warps fold the staged rows (a3) while the K/V stream
 //                  runs.
 //   k_encode_warp  a3 (Sec. 3.3, Eq. (3)) on its own, for ptenc_encode: a warp per (layer, sequence) folds one row --
 //                  the staged one, or a row the caller supplies -- with the routine the attention kernel uses.
