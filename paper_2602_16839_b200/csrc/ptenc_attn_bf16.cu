@@ -292,6 +292,10 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
   // In the common launch -- every entry has tiles and no unit is split -- item i is simply (entry i / H_kv, head
   // i % H_kv), and CTA c starts on item c: the ring words of that entry are requested now, with the first pass.
   const Raw first_raw = fetch((int)blockIdx.x / Hkv);
+  // The producer's first request to the work counter (the number of its second item, or its one failing grab) is
+  // made here as well, so that the answer is there when the first item's tiles have been issued.
+  int first_grab = 0;
+  if (tid == NW * 32) first_grab = atomicAdd(p.work, 1) + (int)gridDim.x;
   long long mine = 0;
   int nz = 0, mx = 0;                                        // entries with tiles, longest entry
 #pragma unroll 1
@@ -501,7 +505,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     } else {
       pd = lookup_begin((int)blockIdx.x);
     }
-    int grabbed = grab();                                    // the item after that; every CTA makes exactly one grab
+    int grabbed = first_grab;                                // the item after that; every CTA makes exactly one grab
                                                              // that finds nothing left (this one, if it has no item)
     while (!aborted) {
       const Item cur = lookup_finish(pd);
