@@ -600,3 +600,34 @@ def test_a_step_with_every_sequence_inactive_changes_nothing_and_leaves_the_coun
             p.step(t)
         assert p.cache.status() == 0
         p.close()
+
+
+@pytest.mark.parametrize("warps", [0, 3])
+def test_item_lookup_by_arithmetic_and_by_search_give_the_same_bits(warps):
+    """The attention kernel finds the (layer, sequence, head) of a work item by arithmetic when every sequence of the
+    call has tokens and no unit is split, and by a search over prefix sums otherwise.  Masking one sequence out
+    switches a launch from the first way to the second; the other sequences' outputs and log-sum-exps must not
+    change by a bit (nor does it matter which CTA a work item lands on)."""
+    L, B, Hq = 2, 6, 8
+    p = Pair(pt, n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=2, head_dim=128, window=200, dtype="bf16", seed=21,
+             attn_consumer_warps=warps)
+    for t in range(230):
+        p.step(t, check=(t % 50 == 0))
+    q = p.gen.step_q(230)
+    out_a = torch.zeros(L, B, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.full_like(out_a, 3.0)
+    lse_a = torch.zeros(L, B, Hq, dtype=torch.float32, device="cuda")
+    lse_b = torch.full_like(lse_a, 3.0)
+    p.cache.decode_attn(-1, q, out_a, None, lse_a)
+    for masked in (0, 3, B - 1):
+        act = torch.ones(B, dtype=torch.uint8, device="cuda")
+        act[masked] = 0
+        out_b.fill_(3.0)
+        lse_b.fill_(3.0)
+        p.cache.decode_attn(-1, q, out_b, act, lse_b)
+        keep = [b for b in range(B) if b != masked]
+        assert torch.equal(out_a[:, keep], out_b[:, keep])
+        assert torch.equal(lse_a[:, keep], lse_b[:, keep])
+        assert torch.equal(out_b[:, masked], torch.full_like(out_b[:, masked], 3.0))      # not written
+    assert p.cache.status() == 0
+    p.close()
