@@ -86,10 +86,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+// Largest K/V volume of a launch whose tile loads carry the L2 "evict first" hint (see ptenc_attn_kv_hint).
+#ifndef PTENC_ATTN_EVICT_FIRST_MAX_BYTES
+#define PTENC_ATTN_EVICT_FIRST_MAX_BYTES (4ull << 30)
+#endif
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// hinted != 0: the copy carries the L2 eviction policy `pol`
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            int hinted, uint64_t pol) {
+  if (hinted) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol) : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+  }
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -181,7 +198,7 @@ template <int D, int TILE_N, int NW, int STAGES, bool SCORE>
 __global__ void __launch_bounds__((NW + 1 + PTENC_ATTN_ENC_WARPS) * 32, PTENC_ATTN_CTAS_PER_SM)
 k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const int l0, const int nl, const __nv_bfloat16* __restrict__ q, const uint8_t* __restrict__ active,
-            __nv_bfloat16* __restrict__ out, float* __restrict__ lse, const int fold_staged) {
+            __nv_bfloat16* __restrict__ out, float* __restrict__ lse, const int fold_staged, const int kv_hint) {
   using SM = Smem<D, TILE_N, NW, STAGES>;
   constexpr int NE = PTENC_ATTN_ENC_WARPS;
   constexpr int NTHREADS = (NW + 1 + NE) * 32;               // consumers, the TMA producer, the encoder warps
@@ -400,6 +417,7 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
     // stages.  One lane issuing every tile of the CTA (a barrier wait, the transaction count and four bulk copies
     // per tile, ~0.3 us) could just keep up with one SM's share of the HBM stream and fell behind at every item
     // boundary; NW lanes in parallel have headroom.
+    const uint64_t kv_policy = l2_evict_first_policy();
     uint32_t kmine = 0;                                      // tiles this lane has issued into its warp's stages
     uint32_t useq = 0;                                       // items handed to the consumers
     bool aborted = false;
@@ -568,8 +586,8 @@ k_attn_bf16(const PtencDev p, const __grid_constant__ CUtensorMap tmK, const __g
           const int y = (int)yy;
 #pragma unroll
           for (int hf = 0; hf < D / 64; ++hf) {
-            tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb);
-            tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb);
+            tma_load_2d(dst + hf * HALF_BYTES, &tmK, hf * 64, y, fb, kv_hint, kv_policy);
+            tma_load_2d(dst + SM::K_BYTES + hf * HALF_BYTES, &tmV, hf * 64, y, fb, kv_hint, kv_policy);
           }
           kmine += 1;
         }
@@ -978,6 +996,17 @@ inline bool use_long_variant(const ptenc_config& cfg, int nl, int tile_n) {
   return cfg.attn_consumer_warps == NW_LONG && NW_LONG != NW_DEFAULT;
 }
 
+// K and V tiles are read once per launch.  Marked "evict first", the tiles of a launch compete only with one another
+// for L2, and what survives to the next step is a part of the rings instead of nothing: a call whose K/V bytes are a
+// few times the 126 MB of L2 finds a part of them there.  Measured, hint on every launch against on none: 0.45 GiB of
+// K/V per step -7.0 % step time, 0.89 GiB -3.3 %, 1.8 GiB -1.4 .. -3.6 %, 2.3 GiB (the 3B shape) -1.9 %, 3.5 GiB
+// -0.4 %, 7 GiB +0.3 %, 14 GiB (the 7B shape) +2.1 %, 28 .. 56 GiB +1 .. 2 %: on the largest calls there is nothing to
+// find and the hinted loads stream a little slower, so the hint is given up to 4 GiB only.
+inline int ptenc_attn_kv_hint(int nl, const ptenc_config& cfg) {
+  const unsigned long long bytes = 2ull * nl * cfg.batch * cfg.n_kv_heads * cfg.window * cfg.head_dim * 2ull;
+  return bytes <= PTENC_ATTN_EVICT_FIRST_MAX_BYTES ? 1 : 0;
+}
+
 template <int D, int NW, bool SCORE>
 cudaError_t launch_ts(ptenc_cache* c, int l0, int nl, const void* q, const uint8_t* active, void* out, float* lse,
                       bool fold_staged, bool early, cudaStream_t st) {
@@ -999,7 +1028,8 @@ cudaError_t launch_ts(ptenc_cache* c, int l0, int nl, const void* q, const uint8
     cfg.numAttrs = 1;
   }
   cudaError_t e = cudaLaunchKernelEx(&cfg, k_attn_bf16<D, TN, NW, STAGES, SCORE>, c->dev, c->tmK, c->tmV, l0, nl,
-                                     (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, fold_staged ? 1 : 0);
+                                     (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, fold_staged ? 1 : 0,
+                                     ptenc_attn_kv_hint(nl, c->cfg));
   c->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -1125,11 +1155,11 @@ cudaError_t static_setup(int device, StaticDevice** out) {
 
 template <int D, int NW>
 cudaError_t launch_static_t(const PtencDev& dev, const CUtensorMap& tmK, const CUtensorMap& tmV, int grid, int nl,
-                            const void* q, const uint8_t* active, void* out, float* lse, cudaStream_t st) {
+                            const void* q, const uint8_t* active, void* out, float* lse, int kv_hint, cudaStream_t st) {
   constexpr int STAGES = Pick<D>::STAGES, TN = Pick<D>::TILE_N;
   using SM = Smem<D, TN, NW, STAGES>;
   k_attn_bf16<D, TN, NW, STAGES, false><<<grid, (NW + 1 + PTENC_ATTN_ENC_WARPS) * 32, SM::TOTAL + 1024, st>>>(
-      dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, 0);
+      dev, tmK, tmV, 0, nl, (const __nv_bfloat16*)q, active, (__nv_bfloat16*)out, lse, 0, kv_hint);
   return cudaGetLastError();
 }
 
@@ -1187,6 +1217,7 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   d.part_slots = STATIC_MAX_SLOTS;
   int grid = sd->sm_count * PTENC_ATTN_CTAS_PER_SM;
   if (2 * grid > STATIC_MAX_SLOTS) grid = STATIC_MAX_SLOTS / 2;
+  const int kv_hint = ptenc_attn_kv_hint(cfg->n_layers, *cfg);
 
   // The array keeps whatever the last call left: the status word, the work counter and the tickets must start at zero.
   if (cudaMemsetAsync(sd->scratch, 0, STATIC_OFF_TICKETS + (size_t)units * 4, st) != cudaSuccess) return PTENC_ECUDA;
@@ -1194,11 +1225,11 @@ extern "C" int ptenc_attn_rings_static(const ptenc_config* cfg, const void* K, c
   const bool lng = use_long_variant(*cfg, cfg->n_layers, tile_n);
   cudaError_t e;
   if (cfg->head_dim == 128)
-    e = lng ? launch_static_t<128, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
-            : launch_static_t<128, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
+    e = lng ? launch_static_t<128, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, kv_hint, st)
+            : launch_static_t<128, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, kv_hint, st);
   else
-    e = lng ? launch_static_t<64, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st)
-            : launch_static_t<64, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, st);
+    e = lng ? launch_static_t<64, NW_LONG>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, kv_hint, st)
+            : launch_static_t<64, NW_DEFAULT>(d, tmK, tmV, grid, cfg->n_layers, q, active, out, lse_out, kv_hint, st);
   if (e != cudaSuccess) return PTENC_ECUDA;
   if (status_out != nullptr &&
       cudaMemcpyAsync(status_out, d.status, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
